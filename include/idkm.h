@@ -1,0 +1,168 @@
+/*
+ * idkm.h -- C ABI of the IDKM hot path on one CUDA device (sm_100a).
+ *
+ * IDKM ("Memory Efficient Neural Network Quantization via Implicit, Differentiable k-Means")
+ * clusters a layer's m weight-vectors w_i in R^d around k = 2^b codewords c_j with a soft,
+ * attention-based k-means (Section 3.2, Algorithm 1), treats the result as the solution of the
+ * fixed-point equation C* = F(C*, W) (Section 4.1) and differentiates it either implicitly
+ * (Section 4.2) or with Jacobian-free backpropagation (Section 4.3).
+ *
+ * Shapes and layout.  All tensors are fp32, row-major, in DEVICE memory unless a parameter says
+ * "host":  W, Wq, dWq, dW are [m][d];  C0, C, dC are [k][d] ([n_layers][k][d] when batched);
+ * A is [m][k].  Every pointer must be 16-byte aligned.  d is 1, 2 or 4; 1 <= k <= 256.
+ *
+ *   D_ij = ||w_i - c_j||_2,  A_ij = softmax_j(-D_ij / tau)            (Algorithm 1, steps 3-4)
+ *   F(C, W)_j = sum_i A_ij w_i / sum_i A_ij                           (Algorithm 1, step 5)
+ *   Wq_i = sum_j A_ij c_j                                             (soft quantiser r_tau)
+ *
+ * Ownership.  The caller owns every buffer, including the workspace; the library borrows them
+ * and allocates no device memory in the device-pointer entry points (idkm_create allocates a few
+ * bytes of bookkeeping on the host only).  Calls are asynchronous on the given CUDA stream.
+ * From idkm_forward* until the matching idkm_backward returns, W, C_out and the workspace must
+ * stay valid and unmodified: the backward recomputes the attention matrix from W and C_out and
+ * reads the column sums and map values stashed in the workspace by the forward's final pass.
+ *
+ * Errors.  Every function returns an int status (IDKM_OK = 0, negative = error) and never
+ * throws, aborts or traps the device.  Argument and launch errors come back synchronously.
+ * Conditions that only the device can see (non-finite values, a diverging adjoint iteration,
+ * the iteration cap reached before the tolerance) are reported in idkm_info.status after
+ * idkm_get_info.
+ */
+#ifndef IDKM_H
+#define IDKM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define IDKM_MAX_K 256
+#define IDKM_MAX_LAYERS 64
+
+/* status codes */
+#define IDKM_OK 0
+#define IDKM_MAXITER 1           /* advisory: iteration cap reached before the tolerance        */
+#define IDKM_ERR_NULL (-1)       /* a required pointer is NULL                                  */
+#define IDKM_ERR_ALIGN (-2)      /* a pointer is not 16-byte aligned                            */
+#define IDKM_ERR_SHAPE (-3)      /* m < 1, bad layer offsets, n_layers out of range             */
+#define IDKM_ERR_UNSUPPORTED (-4)/* d not in {1,2,4} or k not in [1,256]                        */
+#define IDKM_ERR_PARAM (-5)      /* tau <= 0, tol < 0, max_iter < 0, alpha not in (0,1], ...    */
+#define IDKM_ERR_WORKSPACE (-6)  /* workspace smaller than idkm_workspace_bytes()               */
+#define IDKM_ERR_ORDER (-7)      /* idkm_backward without a preceding idkm_forward              */
+#define IDKM_ERR_CUDA (-8)       /* a CUDA runtime call failed                                  */
+#define IDKM_ERR_NONFINITE (-9)  /* device: NaN/Inf met in W, C or the sums                     */
+#define IDKM_ERR_DIVERGED (-10)  /* device: adjoint iteration produced non-finite values or its
+                                    residual grew 10 steps running (Section 4.2: retry with a
+                                    smaller alpha)                                              */
+
+typedef struct idkm_ctx idkm_ctx; /* opaque; remembers the last forward call for the backward */
+
+typedef enum { IDKM_IMPLICIT = 0, IDKM_JFB = 1 } idkm_mode;
+
+/* One record per layer, filled by idkm_get_info. */
+typedef struct {
+  int32_t status;         /* IDKM_OK, IDKM_MAXITER or a device-side error                      */
+  int32_t fwd_iters;      /* applications of F made by the forward loop                        */
+  float   fwd_residual;   /* ||C+ - C||_F / ||C+||_F of the last application                   */
+  int32_t dead_clusters;  /* clusters whose column sum fell below 1e-20 in the last step       */
+  int32_t adj_iters;      /* adjoint iterations made by the last backward                      */
+  float   adj_residual;   /* ||u+ - u||_F / ||u+||_F of the last adjoint iteration             */
+} idkm_info;
+
+/* Create / destroy a context bound to the current CUDA device.  Host allocation only. */
+int  idkm_create(idkm_ctx** out);
+void idkm_destroy(idkm_ctx* ctx);
+
+/* Bytes of device workspace the forward and backward need for a problem of m_total rows in
+ * n_layers layers (1 for the single-layer calls).  Returns 0 for unsupported d or k. */
+size_t idkm_workspace_bytes(int64_t m_total, int d, int k, int n_layers);
+
+/*
+ * Forward: Algorithm 1 (soft k-means) followed by the soft quantiser (Section 3.2).
+ *
+ * Starting from C0, applies C <- F(C, W) until the relative change ||C+ - C||_F / ||C+||_F drops
+ * below tol, or max_iter applications were made (tol = 0: exactly max_iter applications;
+ * max_iter = 0: C_out = C0).  The loop runs on the device: each application is one fused launch
+ * that never stores the m x k attention matrix, and the convergence test is made by the device
+ * without a host round trip (launches queued after convergence return at once).  A cluster whose
+ * column sum is below 1e-20 keeps its centroid.  Then one final pass at the returned centroids
+ * writes Wq = A C (Wq_out, may be NULL), optionally A itself (A_out, may be NULL: m*k floats, the
+ * paper's O(m 2^b) term), and stashes S_j = sum_i A_ij and F(C, W)_j in the workspace.
+ *
+ * C_out receives the last C+ ("return C+", Algorithm 1).  C0 and C_out may alias.
+ */
+int idkm_forward(idkm_ctx* ctx, const float* W, int64_t m, int d, const float* C0, int k, float tau, float tol,
+                 int max_iter, float* C_out, float* A_out, float* Wq_out, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream);
+
+/*
+ * Batched forward: the same for n_layers independent layers that share d, k, tau, tol and
+ * max_iter ("for all layers", Algorithm 2), in the same launches.  W_cat holds the layers' rows
+ * back to back; layer l owns rows [layer_offsets[l], layer_offsets[l+1]) (HOST array of
+ * n_layers+1 increasing int64, first entry 0); C0 / C_out are [n_layers][k][d]; A_out / Wq_out
+ * follow W_cat's row order.  Each layer converges (and stops being touched) on its own.
+ * 1 <= n_layers <= IDKM_MAX_LAYERS.
+ */
+int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer_offsets, int n_layers, int d,
+                         const float* C0, int k, float tau, float tol, int max_iter, float* C_out, float* A_out,
+                         float* Wq_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/*
+ * Backward of L = <dWq, Wq(W, C*(W))> at the centroids returned by the last forward of this ctx.
+ *
+ * IDKM_IMPLICIT (Section 4.2): solves u = J_C^T u + g, J_C = dF/dC, by the averaged iteration
+ *   u <- alpha (J_C^T u + g) + (1 - alpha) u from u = g, until the relative change of u is below
+ *   adj_tol or adj_max_iter steps were made (adj_tol = 0: exactly adj_max_iter steps).  This is
+ *   the vector form of the paper's iteration M <- alpha ((dF/dC) M + I) + (1 - alpha) M for
+ *   M* = (I - dF/dC)^-1, contracted with g (u* = M*^T g); alpha = 1 is the plain iteration, the
+ *   paper uses 0.25.  Each step is one fused vector-Jacobian pass over W; nothing is stored per step.
+ * IDKM_JFB (Section 4.3): M* = I, i.e. u = g and no adjoint iterations.
+ *
+ * g = (dWq/dC)^T dWq is the direct codebook gradient.  Outputs:
+ *   dW_out [m][d] = (dWq/dW)^T dWq + (dF/dW)^T u     (may be NULL)
+ *   dC_out [k][d] ([n_layers][k][d]) = u             (may be NULL)
+ * dWq has W's shape; dW_out must not alias dWq or W.  workspace must be the forward's.
+ */
+int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol, int adj_max_iter, float alpha,
+                  float* dW_out, float* dC_out, void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Waits for the ctx's stream and copies one idkm_info per layer of the last forward to the HOST
+ * array info_out (n_layers entries; 1 for idkm_forward). */
+int idkm_get_info(idkm_ctx* ctx, idkm_info* info_out);
+
+/*
+ * Whole hot path on HOST buffers (Algorithm 2's per-layer work: cluster, quantise, differentiate):
+ * copies W, C0 and dWq to the device, runs idkm_forward_batched and idkm_backward, and copies
+ * C, Wq, dW, dC back; returns after everything has completed.  Device buffers are allocated on
+ * first use, kept in the ctx and grown on demand (this is the only entry point that allocates
+ * device memory).  Any of Wq_out, dW_out, dC_out may be NULL; info_out (n_layers entries) too.
+ * layer_offsets as in idkm_forward_batched (pass {0, m} and n_layers = 1 for one layer).
+ */
+int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
+                       const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
+                       idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
+                       float* Wq_out_host, float* dW_out_host, float* dC_out_host, idkm_info* info_out);
+
+/*
+ * Phase timing.  idkm_set_timing(ctx, 1) makes the following forward / backward calls record CUDA
+ * events on their stream between phases (a few microseconds per call; events are created on the
+ * first enable).  idkm_get_phase_ms waits for the last recorded call and writes six elapsed times in
+ * milliseconds to the HOST array ms_out: [0] state initialisation, [1] the loop of fused forward
+ * steps (Algorithm 1), [2] the final pass, [3] the direct codebook-gradient pass, [4] the loop of
+ * adjoint steps (Section 4.2), [5] the pass that writes dL/dW.  A phase that has not run is -1.
+ */
+int idkm_set_timing(idkm_ctx* ctx, int enable);
+int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out);
+
+/* Number of kernels this ctx has launched since idkm_create (for accounting in benchmarks). */
+int64_t idkm_launch_count(const idkm_ctx* ctx);
+
+/* Static, human-readable text for a status code. */
+const char* idkm_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IDKM_H */

@@ -1,0 +1,513 @@
+// Host side of the C ABI declared in include/idkm.h: argument checks, workspace layout, tile
+// tables and the launch sequences.  Every step of the path runs in the kernels of
+// idkm_kernels.cuh; nothing here computes on the data.
+#include "idkm_kernels.cuh"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/idkm.h"
+
+namespace idkm {
+
+extern const KernelEntry k_table_step[3][N_FAMILY];
+extern const KernelEntry k_table_final[3][N_FAMILY];
+extern const KernelEntry k_table_grad[3][N_FAMILY];
+extern const KernelEntry k_table_adj[3][N_FAMILY];
+extern const KernelEntry k_table_scatter[3][N_FAMILY];
+extern const KernelEntry k_table_step_precise[3][N_FAMILY];
+
+// Initialise the per-layer state and copy C0 into the working centroids.
+__global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
+                                  double inv_tau) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_layers) {
+    LayerState s;
+    s.fwd_done = 0; s.fwd_iters = 0; s.fwd_res = 0.f; s.dead = 0;
+    s.adj_done = 0; s.adj_iters = 0; s.adj_res = 0.f; s.status = ST_OK;
+    s.ticket = 0u; s.adj_up = 0; s.adj_prev = 3.0e38f;
+    for (int q = 0; q < 4; ++q) s.pad[q] = 0;
+    // bounding box of the starting centroids decides which step kernel takes the layer first
+    double box2 = 0.0;
+    for (int a = 0; a < d; ++a) {
+      double lo = 1e300, hi = -1e300;
+      for (int j = 0; j < k; ++j) {
+        const double v = (double)C0[((size_t)i * k + j) * d + a];
+        lo = fmin(lo, v);
+        hi = fmax(hi, v);
+      }
+      box2 += (hi - lo) * (hi - lo);
+    }
+    s.precise = (sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
+    st[i] = s;
+  }
+  if (C0 != C)
+    for (int o = i; o < n_coord; o += gridDim.x * blockDim.x) C[o] = C0[o];
+}
+
+static int d_index(int d) { return d == 1 ? 0 : (d == 2 ? 1 : (d == 4 ? 2 : -1)); }
+
+const KernelEntry* kernel_entry(int mode, int d, int family) {
+  const int di = d_index(d);
+  if (di < 0 || family < 0 || family >= N_FAMILY) return nullptr;
+  switch (mode) {
+    case STEP: return &k_table_step[di][family];
+    case FINAL: return &k_table_final[di][family];
+    case GRAD: return &k_table_grad[di][family];
+    case ADJ: return &k_table_adj[di][family];
+    case SCATTER: return &k_table_scatter[di][family];
+    case STEP_PRECISE: return &k_table_step_precise[di][family];
+  }
+  return nullptr;
+}
+
+int pick_family(int mode, int d, int k) {
+  for (int f = 0; f < N_FAMILY; ++f) {
+    const KernelEntry* e = kernel_entry(mode, d, f);
+    if (e && e->kpl * e->lpw >= k) return f;
+  }
+  return -1;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct WorkspaceLayout {
+  size_t off_state, off_S, off_F, off_g, off_u, off_partials, total;
+  int max_slots;
+};
+
+static int device_sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      sms <= 0) {
+    (void)cudaGetLastError();
+    return 148;
+  }
+  return sms;
+}
+
+static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* out) {
+  if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K || n_layers < 1 || n_layers > IDKM_MAX_LAYERS) return false;
+  int plen_max = 1;
+  for (int mode = STEP; mode < N_MODES; ++mode) {
+    const int f = pick_family(mode, d, k);
+    if (f < 0) return false;
+    const int pl = kernel_entry(mode, d, f)->plen;
+    if (pl > plen_max) plen_max = pl;
+  }
+  WorkspaceLayout w;
+  size_t o = 0;
+  w.off_state = o; o = align_up(o + sizeof(LayerState) * (size_t)n_layers, 256);
+  w.off_S = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k, 256);
+  w.off_F = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k * d, 256);
+  w.off_g = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k * d, 256);
+  w.off_u = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k * d, 256);
+  w.max_slots = sms * MAX_BLOCKS_PER_SM + n_layers;
+  w.off_partials = o; o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen_max, 256);
+  w.total = o;
+  *out = w;
+  return true;
+}
+
+}  // namespace idkm
+
+using namespace idkm;
+
+struct idkm_ctx {
+  int device;
+  int sms;
+  int64_t launches;
+  // last forward
+  bool have_forward;
+  const float* W;
+  float* C;
+  void* workspace;
+  int64_t m_total;
+  int d, k, n_layers;
+  float tau;
+  long long row_off[MAX_LAYERS + 1];
+  cudaStream_t stream;
+  int occupancy[N_MODES][3][N_FAMILY];   // cached blocks/SM per kernel, 0 = not queried
+  // device buffers of the host-pointer entry point
+  void* hbuf;
+  size_t hbuf_bytes;
+  // optional phase timing (CUDA events on the call's stream)
+  bool timing;
+  bool ev_ok;
+  bool ev_fwd_set, ev_bwd_set;
+  cudaEvent_t ev[8];   // fwd: 0 start, 1 after init, 2 after steps, 3 after final; bwd: 4 start, 5 grad, 6 adj, 7 scatter
+};
+
+static void mark(idkm_ctx* ctx, int i) {
+  if (ctx->timing && ctx->ev_ok) cudaEventRecord(ctx->ev[i], ctx->stream);
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int blocks_per_sm(idkm_ctx* ctx, int mode, int d, int family) {
+  int& slot = ctx->occupancy[mode][d_index(d)][family];
+  if (slot == 0) {
+    int n = 0;
+    const KernelEntry* e = kernel_entry(mode, d, family);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, e->func, BLOCK, 0) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      n = 1;
+    }
+    slot = n > MAX_BLOCKS_PER_SM ? MAX_BLOCKS_PER_SM : n;
+  }
+  return slot;
+}
+
+// Tile table of one pass: tiles never span layers; blocks get contiguous tile ranges.
+static int build_table(idkm_ctx* ctx, int mode, int family, LayerTable* lt) {
+  const KernelEntry* e = kernel_entry(mode, ctx->d, family);
+  lt->n_layers = ctx->n_layers;
+  long long tiles = 0;
+  for (int l = 0; l < ctx->n_layers; ++l) {
+    lt->row_off[l] = ctx->row_off[l];
+    lt->tile_off[l] = (int)tiles;
+    const long long rows = ctx->row_off[l + 1] - ctx->row_off[l];
+    tiles += (rows + e->tile - 1) / e->tile;
+    if (tiles > 0x7fffffffLL / 2) return IDKM_ERR_SHAPE;
+  }
+  lt->row_off[ctx->n_layers] = ctx->row_off[ctx->n_layers];
+  lt->tile_off[ctx->n_layers] = (int)tiles;
+  for (int l = ctx->n_layers + 1; l <= MAX_LAYERS; ++l) {
+    lt->row_off[l] = lt->row_off[ctx->n_layers];
+    lt->tile_off[l] = 0x7fffffff;
+  }
+  lt->tiles_total = (int)tiles;
+  long long nb = (long long)ctx->sms * blocks_per_sm(ctx, mode, ctx->d, family);
+  if (nb > tiles) nb = tiles;
+  lt->n_blocks = (int)nb;
+  lt->pad = 0;
+  return IDKM_OK;
+}
+
+static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p) {
+  memset(p, 0, sizeof(*p));
+  char* ws = static_cast<char*>(ctx->workspace);
+  p->W = ctx->W;
+  p->C = ctx->C;
+  p->S = reinterpret_cast<float*>(ws + wl.off_S);
+  p->F = reinterpret_cast<float*>(ws + wl.off_F);
+  p->gvec = reinterpret_cast<float*>(ws + wl.off_g);
+  p->u = reinterpret_cast<float*>(ws + wl.off_u);
+  p->partials = reinterpret_cast<double*>(ws + wl.off_partials);
+  p->st = reinterpret_cast<LayerState*>(ws + wl.off_state);
+  p->inv_tau = (float)(1.0 / (double)ctx->tau);
+  p->inv_tau_d = 1.0 / (double)ctx->tau;
+  p->scale = (float)(1.4426950408889634 / (double)ctx->tau);
+  p->alpha = 1.f;
+  p->k = ctx->k;
+}
+
+// The forward loop: every iteration launches the fp32 step and the fp64 step; each layer is taken by exactly one
+// of them (LayerState::precise), the other returns at once for it.
+static int launch_step_loop(idkm_ctx* ctx, PassParams* p, int repeat) {
+  const int f32 = pick_family(STEP, ctx->d, ctx->k), f64 = pick_family(STEP_PRECISE, ctx->d, ctx->k);
+  const KernelEntry* e32 = kernel_entry(STEP, ctx->d, f32);
+  const KernelEntry* e64 = kernel_entry(STEP_PRECISE, ctx->d, f64);
+  PassParams q = *p;
+  int rc = build_table(ctx, STEP, f32, &p->lt);
+  if (rc != IDKM_OK) return rc;
+  rc = build_table(ctx, STEP_PRECISE, f64, &q.lt);
+  if (rc != IDKM_OK) return rc;
+  for (int it = 0; it < repeat; ++it) {
+    p->iter = q.iter = it;
+    if (e32->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+    if (e64->launch(q, q.lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+    ctx->launches += 2;
+  }
+  return IDKM_OK;
+}
+
+static int launch_pass(idkm_ctx* ctx, int mode, PassParams* p, int repeat) {
+  const int f = pick_family(mode, ctx->d, ctx->k);
+  const KernelEntry* e = kernel_entry(mode, ctx->d, f);
+  const int rc = build_table(ctx, mode, f, &p->lt);
+  if (rc != IDKM_OK) return rc;
+  for (int it = 0; it < repeat; ++it) {
+    if (e->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+    ++ctx->launches;
+  }
+  return IDKM_OK;
+}
+
+extern "C" {
+
+int idkm_create(idkm_ctx** out) {
+  if (!out) return IDKM_ERR_NULL;
+  idkm_ctx* c = new (std::nothrow) idkm_ctx;
+  if (!c) return IDKM_ERR_CUDA;
+  memset(c, 0, sizeof(*c));
+  if (cudaGetDevice(&c->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->sms, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess || c->sms < 1) {
+    (void)cudaGetLastError();
+    delete c;
+    return IDKM_ERR_CUDA;
+  }
+  *out = c;
+  return IDKM_OK;
+}
+
+void idkm_destroy(idkm_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->hbuf) cudaFree(ctx->hbuf);
+  if (ctx->ev_ok)
+    for (int i = 0; i < 8; ++i) cudaEventDestroy(ctx->ev[i]);
+  delete ctx;
+}
+
+size_t idkm_workspace_bytes(int64_t m_total, int d, int k, int n_layers) {
+  WorkspaceLayout wl;
+  if (m_total < 1 || !make_layout(d, k, n_layers, device_sm_count(), &wl)) return 0;
+  return wl.total;
+}
+
+int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer_offsets, int n_layers, int d,
+                         const float* C0, int k, float tau, float tol, int max_iter, float* C_out, float* A_out,
+                         float* Wq_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !W_cat || !layer_offsets || !C0 || !C_out || !workspace) return IDKM_ERR_NULL;
+  if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K) return IDKM_ERR_UNSUPPORTED;
+  if (n_layers < 1 || n_layers > IDKM_MAX_LAYERS) return IDKM_ERR_SHAPE;
+  if (layer_offsets[0] != 0) return IDKM_ERR_SHAPE;
+  for (int l = 0; l < n_layers; ++l)
+    if (layer_offsets[l + 1] <= layer_offsets[l]) return IDKM_ERR_SHAPE;
+  const int64_t m_total = layer_offsets[n_layers];
+  if (m_total < 1 || m_total > (1LL << 40) / (k > d ? k : d)) return IDKM_ERR_SHAPE;
+  if (!(tau > 0.f) || !isfinite(tau) || !(tol >= 0.f) || !isfinite(tol) || max_iter < 0) return IDKM_ERR_PARAM;
+  if (!aligned16(W_cat) || !aligned16(C0) || !aligned16(C_out) || !aligned16(workspace) ||
+      (A_out && !aligned16(A_out)) || (Wq_out && !aligned16(Wq_out)))
+    return IDKM_ERR_ALIGN;
+  WorkspaceLayout wl;
+  if (!make_layout(d, k, n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (workspace_bytes < wl.total) return IDKM_ERR_WORKSPACE;
+
+  ctx->have_forward = false;
+  ctx->W = W_cat;
+  ctx->C = C_out;
+  ctx->workspace = workspace;
+  ctx->m_total = m_total;
+  ctx->d = d;
+  ctx->k = k;
+  ctx->n_layers = n_layers;
+  ctx->tau = tau;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+  for (int l = 0; l <= n_layers; ++l) ctx->row_off[l] = layer_offsets[l];
+
+  PassParams p;
+  fill_params(ctx, wl, &p);
+  p.tol = tol;
+  p.max_iter = max_iter;
+
+  ctx->ev_fwd_set = ctx->ev_bwd_set = false;
+  mark(ctx, 0);
+  const int n_coord = n_layers * k * d;
+  const int init_threads = n_coord > n_layers ? n_coord : n_layers;
+  idkm_init_forward<<<(init_threads + 255) / 256, 256, 0, ctx->stream>>>(p.st, n_layers, C0, C_out, n_coord, k, d,
+                                                                                     p.inv_tau_d);
+  if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
+  ++ctx->launches;
+  mark(ctx, 1);
+
+  int rc = launch_step_loop(ctx, &p, max_iter);
+  if (rc != IDKM_OK) return rc;
+  mark(ctx, 2);
+  p.Wq = Wq_out;
+  p.A = A_out;
+  rc = launch_pass(ctx, FINAL, &p, 1);
+  if (rc != IDKM_OK) return rc;
+  mark(ctx, 3);
+  ctx->ev_fwd_set = ctx->timing && ctx->ev_ok;
+  ctx->have_forward = true;
+  return IDKM_OK;
+}
+
+int idkm_forward(idkm_ctx* ctx, const float* W, int64_t m, int d, const float* C0, int k, float tau, float tol,
+                 int max_iter, float* C_out, float* A_out, float* Wq_out, void* workspace, size_t workspace_bytes,
+                 void* cuda_stream) {
+  if (m < 1) return ctx ? IDKM_ERR_SHAPE : IDKM_ERR_NULL;
+  const int64_t offs[2] = {0, m};
+  return idkm_forward_batched(ctx, W, offs, 1, d, C0, k, tau, tol, max_iter, C_out, A_out, Wq_out, workspace,
+                              workspace_bytes, cuda_stream);
+}
+
+int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol, int adj_max_iter, float alpha,
+                  float* dW_out, float* dC_out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!ctx || !dWq || !workspace) return IDKM_ERR_NULL;
+  if (!ctx->have_forward) return IDKM_ERR_ORDER;
+  if (workspace != ctx->workspace) return IDKM_ERR_ORDER;
+  if (mode != IDKM_IMPLICIT && mode != IDKM_JFB) return IDKM_ERR_PARAM;
+  if (!(adj_tol >= 0.f) || !isfinite(adj_tol) || adj_max_iter < 0 || !(alpha > 0.f) || !(alpha <= 1.f))
+    return IDKM_ERR_PARAM;
+  if (!aligned16(dWq) || (dW_out && !aligned16(dW_out)) || (dC_out && !aligned16(dC_out))) return IDKM_ERR_ALIGN;
+  if (dW_out && (dW_out == dWq || dW_out == ctx->W)) return IDKM_ERR_PARAM;
+  WorkspaceLayout wl;
+  if (!make_layout(ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (workspace_bytes < wl.total) return IDKM_ERR_WORKSPACE;
+  ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+
+  PassParams p;
+  fill_params(ctx, wl, &p);
+  p.G = dWq;
+  p.tol = adj_tol;
+  p.max_iter = adj_max_iter;
+  p.alpha = alpha;
+  ctx->ev_bwd_set = false;
+  mark(ctx, 4);
+  int rc = launch_pass(ctx, GRAD, &p, 1);
+  if (rc != IDKM_OK) return rc;
+  mark(ctx, 5);
+  if (mode == IDKM_IMPLICIT) {
+    rc = launch_pass(ctx, ADJ, &p, adj_max_iter);
+    if (rc != IDKM_OK) return rc;
+  }
+  mark(ctx, 6);
+  if (dW_out) {
+    p.dW = dW_out;
+    rc = launch_pass(ctx, SCATTER, &p, 1);
+    if (rc != IDKM_OK) return rc;
+  }
+  mark(ctx, 7);
+  ctx->ev_bwd_set = ctx->timing && ctx->ev_ok;
+  if (dC_out) {
+    if (cudaMemcpyAsync(dC_out, p.u, sizeof(float) * (size_t)ctx->n_layers * ctx->k * ctx->d, cudaMemcpyDeviceToDevice,
+                        ctx->stream) != cudaSuccess)
+      return IDKM_ERR_CUDA;
+  }
+  return IDKM_OK;
+}
+
+int idkm_get_info(idkm_ctx* ctx, idkm_info* info_out) {
+  if (!ctx || !info_out) return IDKM_ERR_NULL;
+  if (!ctx->have_forward) return IDKM_ERR_ORDER;
+  WorkspaceLayout wl;
+  if (!make_layout(ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  LayerState host[MAX_LAYERS];
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (cudaMemcpy(host, static_cast<char*>(ctx->workspace) + wl.off_state, sizeof(LayerState) * (size_t)ctx->n_layers,
+                 cudaMemcpyDeviceToHost) != cudaSuccess)
+    return IDKM_ERR_CUDA;
+  for (int l = 0; l < ctx->n_layers; ++l) {
+    info_out[l].status = host[l].status;
+    info_out[l].fwd_iters = host[l].fwd_iters;
+    info_out[l].fwd_residual = host[l].fwd_res;
+    info_out[l].dead_clusters = host[l].dead;
+    info_out[l].adj_iters = host[l].adj_iters;
+    info_out[l].adj_residual = host[l].adj_res;
+  }
+  return IDKM_OK;
+}
+
+int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
+                       const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
+                       idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
+                       float* Wq_out_host, float* dW_out_host, float* dC_out_host, idkm_info* info_out) {
+  if (!ctx || !W_host || !layer_offsets || !C0_host || !dWq_host || !C_out_host) return IDKM_ERR_NULL;
+  if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K) return IDKM_ERR_UNSUPPORTED;
+  if (n_layers < 1 || n_layers > IDKM_MAX_LAYERS || layer_offsets[0] != 0) return IDKM_ERR_SHAPE;
+  const int64_t m = layer_offsets[n_layers];
+  if (m < 1) return IDKM_ERR_SHAPE;
+  const size_t ws_bytes = idkm_workspace_bytes(m, d, k, n_layers);
+  if (ws_bytes == 0) return IDKM_ERR_UNSUPPORTED;
+  const size_t wbytes = align_up(sizeof(float) * (size_t)m * d, 256);
+  const size_t cbytes = align_up(sizeof(float) * (size_t)n_layers * k * d, 256);
+  // W, G, Wq, dW | C0, C, dC | workspace
+  const size_t need = 4 * wbytes + 3 * cbytes + align_up(ws_bytes, 256);
+  if (need > ctx->hbuf_bytes) {
+    if (ctx->hbuf) cudaFree(ctx->hbuf);
+    ctx->hbuf = nullptr;
+    ctx->hbuf_bytes = 0;
+    if (cudaMalloc(&ctx->hbuf, need) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return IDKM_ERR_CUDA;
+    }
+    ctx->hbuf_bytes = need;
+  }
+  char* base = static_cast<char*>(ctx->hbuf);
+  float* dW_ = reinterpret_cast<float*>(base);
+  float* dG = reinterpret_cast<float*>(base + wbytes);
+  float* dWq = reinterpret_cast<float*>(base + 2 * wbytes);
+  float* ddW = reinterpret_cast<float*>(base + 3 * wbytes);
+  float* dC0 = reinterpret_cast<float*>(base + 4 * wbytes);
+  float* dC = reinterpret_cast<float*>(base + 4 * wbytes + cbytes);
+  float* ddC = reinterpret_cast<float*>(base + 4 * wbytes + 2 * cbytes);
+  void* ws = base + 4 * wbytes + 3 * cbytes;
+  cudaStream_t s = 0;
+  const size_t wn = sizeof(float) * (size_t)m * d, cn = sizeof(float) * (size_t)n_layers * k * d;
+  if (cudaMemcpyAsync(dW_, W_host, wn, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dC0, C0_host, cn, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+      cudaMemcpyAsync(dG, dWq_host, wn, cudaMemcpyHostToDevice, s) != cudaSuccess)
+    return IDKM_ERR_CUDA;
+  int rc = idkm_forward_batched(ctx, dW_, layer_offsets, n_layers, d, dC0, k, tau, tol, max_iter, dC, nullptr,
+                                Wq_out_host ? dWq : nullptr, ws, ws_bytes, s);
+  if (rc != IDKM_OK) return rc;
+  rc = idkm_backward(ctx, dG, mode, adj_tol, adj_max_iter, alpha, dW_out_host ? ddW : nullptr,
+                     dC_out_host ? ddC : nullptr, ws, ws_bytes, s);
+  if (rc != IDKM_OK) return rc;
+  if (cudaMemcpyAsync(C_out_host, dC, cn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (Wq_out_host && cudaMemcpyAsync(Wq_out_host, dWq, wn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (dW_out_host && cudaMemcpyAsync(dW_out_host, ddW, wn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (dC_out_host && cudaMemcpyAsync(dC_out_host, ddC, cn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (info_out) return idkm_get_info(ctx, info_out);
+  return IDKM_OK;
+}
+
+int idkm_set_timing(idkm_ctx* ctx, int enable) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (enable && !ctx->ev_ok) {
+    for (int i = 0; i < 8; ++i)
+      if (cudaEventCreate(&ctx->ev[i]) != cudaSuccess) {
+        for (int q = 0; q < i; ++q) cudaEventDestroy(ctx->ev[q]);
+        (void)cudaGetLastError();
+        return IDKM_ERR_CUDA;
+      }
+    ctx->ev_ok = true;
+  }
+  ctx->timing = enable != 0;
+  ctx->ev_fwd_set = ctx->ev_bwd_set = false;
+  return IDKM_OK;
+}
+
+int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out) {
+  if (!ctx || !ms_out) return IDKM_ERR_NULL;
+  for (int i = 0; i < 6; ++i) ms_out[i] = -1.f;
+  if (ctx->ev_fwd_set) {
+    if (cudaEventSynchronize(ctx->ev[3]) != cudaSuccess) return IDKM_ERR_CUDA;
+    for (int i = 0; i < 3; ++i)
+      if (cudaEventElapsedTime(&ms_out[i], ctx->ev[i], ctx->ev[i + 1]) != cudaSuccess) return IDKM_ERR_CUDA;
+  }
+  if (ctx->ev_bwd_set) {
+    if (cudaEventSynchronize(ctx->ev[7]) != cudaSuccess) return IDKM_ERR_CUDA;
+    for (int i = 0; i < 3; ++i)
+      if (cudaEventElapsedTime(&ms_out[3 + i], ctx->ev[4 + i], ctx->ev[5 + i]) != cudaSuccess) return IDKM_ERR_CUDA;
+  }
+  return IDKM_OK;
+}
+
+int64_t idkm_launch_count(const idkm_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* idkm_status_string(int status) {
+  switch (status) {
+    case IDKM_OK: return "ok";
+    case IDKM_MAXITER: return "iteration cap reached before the tolerance";
+    case IDKM_ERR_NULL: return "required pointer is NULL";
+    case IDKM_ERR_ALIGN: return "pointer is not 16-byte aligned";
+    case IDKM_ERR_SHAPE: return "bad shape or layer offsets";
+    case IDKM_ERR_UNSUPPORTED: return "unsupported d or k";
+    case IDKM_ERR_PARAM: return "parameter out of range";
+    case IDKM_ERR_WORKSPACE: return "workspace too small";
+    case IDKM_ERR_ORDER: return "backward without a matching forward";
+    case IDKM_ERR_CUDA: return "CUDA runtime error";
+    case IDKM_ERR_NONFINITE: return "non-finite value met on the device";
+    case IDKM_ERR_DIVERGED: return "adjoint iteration diverged";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

@@ -1,0 +1,51 @@
+// Instantiates every (d, codebook layout) variant of one pass and exports its dispatch table.
+// Included by one translation unit per pass so that the units compile in parallel.
+#pragma once
+#include "idkm_kernels.cuh"
+
+namespace idkm {
+
+template <int MODE, int D, int KPL, int LPW>
+static cudaError_t launch_one(const PassParams& p, int grid, cudaStream_t stream) {
+  idkm_pass<MODE, D, KPL, LPW><<<grid, BLOCK, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+
+#define IDKM_ENTRY(MODE, D, KPL, LPW)                                                             \
+  {                                                                                               \
+    &launch_one<MODE, D, KPL, LPW>, (const void*)&idkm_pass<MODE, D, KPL, LPW>, KPL, LPW,         \
+        PassCfg<MODE, D, KPL, LPW>::TILE, PassCfg<MODE, D, KPL, LPW>::PLEN                        \
+  }
+
+template <int D, int KPL, int LPW>
+static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t stream) {
+  idkm_step_precise<D, KPL, LPW><<<grid, BLOCK, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+#define IDKM_PRECISE_ENTRY(D, KPL, LPW)                                                           \
+  {                                                                                               \
+    &launch_precise<D, KPL, LPW>, (const void*)&idkm_step_precise<D, KPL, LPW>, KPL, LPW,         \
+        PreciseCfg<D, KPL, LPW>::TILE, PreciseCfg<D, KPL, LPW>::PLEN                              \
+  }
+#define IDKM_PRECISE_ROW(D)                                                                       \
+  {                                                                                               \
+    IDKM_PRECISE_ENTRY(D, 2, 1), IDKM_PRECISE_ENTRY(D, 4, 1), IDKM_PRECISE_ENTRY(D, 8, 1),        \
+        IDKM_PRECISE_ENTRY(D, 8, 2), IDKM_PRECISE_ENTRY(D, 8, 4), IDKM_PRECISE_ENTRY(D, 8, 8),    \
+        IDKM_PRECISE_ENTRY(D, 8, 16), IDKM_PRECISE_ENTRY(D, 8, 32)                                \
+  }
+
+// forward passes keep 16 centroids per lane, backward passes 8 (they also hold F_j and u_j/S_j)
+#define IDKM_FWD_ROW(MODE, D)                                                                     \
+  {                                                                                               \
+    IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
+        IDKM_ENTRY(MODE, D, 16, 1), IDKM_ENTRY(MODE, D, 16, 2), IDKM_ENTRY(MODE, D, 16, 4),       \
+        IDKM_ENTRY(MODE, D, 16, 8), IDKM_ENTRY(MODE, D, 16, 16)                                   \
+  }
+#define IDKM_BWD_ROW(MODE, D)                                                                     \
+  {                                                                                               \
+    IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
+        IDKM_ENTRY(MODE, D, 8, 2), IDKM_ENTRY(MODE, D, 8, 4), IDKM_ENTRY(MODE, D, 8, 8),          \
+        IDKM_ENTRY(MODE, D, 8, 16), IDKM_ENTRY(MODE, D, 8, 32)                                    \
+  }
+
+}  // namespace idkm

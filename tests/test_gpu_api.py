@@ -1,0 +1,90 @@
+"""Argument checking and host-buffer entry point of the C-ABI library (B200 only)."""
+import numpy as np
+import pytest
+
+from paper_2312_07759_b200 import workloads as WL
+from parity_util import TOL_C, TOL_GRAD, assert_close, oracle_run
+
+pytestmark = pytest.mark.gpu
+
+
+def test_argument_errors():
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    ctx = B.Context()
+    dev = torch.device("cuda:0")
+    W = torch.zeros(1024, 1, device=dev)
+    C0 = torch.zeros(4, 1, device=dev)
+    Co = torch.zeros(4, 1, device=dev)
+    nbytes = B.workspace_bytes(1024, 1, 4, 1)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    args = dict(W=W.data_ptr(), m=1024, d=1, C0=C0.data_ptr(), k=4, tau=0.1, tol=0.0, max_iter=2,
+                C_out=Co.data_ptr(), A_out=None, Wq_out=None, ws=ws.data_ptr(), ws_bytes=nbytes)
+
+    def fwd(**kw):
+        a = dict(args)
+        a.update(kw)
+        return ctx.forward_raw(**a)
+
+    # backward before any forward
+    assert ctx.backward_raw(W.data_ptr(), B.IMPLICIT, 0.0, 1, 1.0, None, None, ws.data_ptr(), nbytes) == B.ERR_ORDER
+    assert fwd(W=None) == B.ERR_NULL
+    assert fwd(W=W.data_ptr() + 4) == B.ERR_ALIGN
+    assert fwd(m=0) == B.ERR_SHAPE
+    assert fwd(d=3) == B.ERR_UNSUPPORTED
+    assert fwd(k=257) == B.ERR_UNSUPPORTED
+    assert fwd(k=0) == B.ERR_UNSUPPORTED
+    assert fwd(tau=0.0) == B.ERR_PARAM
+    assert fwd(tau=float("nan")) == B.ERR_PARAM
+    assert fwd(tol=-1.0) == B.ERR_PARAM
+    assert fwd(max_iter=-1) == B.ERR_PARAM
+    assert fwd(ws_bytes=nbytes - 1) == B.ERR_WORKSPACE
+    assert fwd() == B.OK
+    G = torch.zeros(1024, 1, device=dev)
+    dW = torch.zeros(1024, 1, device=dev)
+    bw = lambda **kw: ctx.backward_raw(**{**dict(dWq=G.data_ptr(), mode=B.IMPLICIT, adj_tol=0.0, adj_max_iter=1,
+                                                 alpha=1.0, dW_out=dW.data_ptr(), dC_out=None, ws=ws.data_ptr(),
+                                                 ws_bytes=nbytes), **kw})
+    assert bw(alpha=0.0) == B.ERR_PARAM
+    assert bw(alpha=1.5) == B.ERR_PARAM
+    assert bw(mode=7) == B.ERR_PARAM
+    assert bw(dW_out=G.data_ptr()) == B.ERR_PARAM
+    assert bw(adj_max_iter=-2) == B.ERR_PARAM
+    assert bw() == B.OK
+    torch.cuda.synchronize()
+    assert B.workspace_bytes(10, 3, 4, 1) == 0
+    assert "workspace" in B.status_string(B.ERR_WORKSPACE)
+
+
+def test_quantize_host_matches_oracle():
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(50000, 2, 16, 0.012, std=0.03, seed=3, max_iter=10, adj_max_iter=6, init="rows")
+    ctx = B.Context()
+    for _ in range(2):   # second call reuses the device buffers
+        C, Wq, dW, dC, infos = ctx.quantize_host(wl.W, wl.C0, wl.G, wl.tau, 0.0, wl.max_iter, B.IMPLICIT, 0.0,
+                                                 wl.adj_max_iter, 1.0)
+        ref = oracle_run(wl)
+        assert infos[0].status == 0 and infos[0].fwd_iters == 10 and infos[0].adj_iters == 6
+        assert_close(C, ref["C"], TOL_C, "C")
+        assert_close(Wq, ref["Wq"], TOL_C, "Wq")
+        assert_close(dW, ref["dW"], TOL_GRAD, "dW")
+        assert_close(dC, ref["dC"], TOL_GRAD, "dC")
+    assert ctx.launches == 2 * (1 + 2 * 10 + 1 + 1 + 6 + 1)   # init, fp32+fp64 step per iteration, final, g, adjoint, dW
+
+
+def test_non_default_stream():
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(10000, 1, 8, 0.01, std=0.03, seed=4, max_iter=8, adj_max_iter=4)
+    ref = oracle_run(wl)
+    s = torch.cuda.Stream()
+    ctx = B.Context()
+    with torch.cuda.stream(s):
+        W = torch.from_numpy(wl.W).cuda()
+        C0 = torch.from_numpy(wl.C0).cuda()
+        G = torch.from_numpy(wl.G).cuda()
+        fr = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter)
+        dW, dC = ctx.backward(G, B.IMPLICIT, 0.0, wl.adj_max_iter, 1.0)
+    s.synchronize()
+    assert_close(fr.C.cpu().numpy(), ref["C"], TOL_C, "C")
+    assert_close(dW.cpu().numpy(), ref["dW"], TOL_GRAD, "dW")

@@ -1,0 +1,215 @@
+"""CUDA path vs float64 oracle, element by element, through the C-ABI library (B200 only)."""
+import numpy as np
+import pytest
+
+from paper_2312_07759_b200 import workloads as WL
+from parity_util import (TOL_C, TOL_GRAD, assert_close, assert_grad_close, at_centroids, gpu_run, kink_crossings, oracle_backward_at,
+                         oracle_run, rel_err)
+
+pytestmark = pytest.mark.gpu
+
+
+# With scalar weights (d = 1) the gradient is a discontinuous function of the centroids: n_ij = sign(w_i - c_j)
+# flips when a centroid moves across a weight.  The chained run (GPU backward at the GPU's own centroids, which
+# agree with the oracle's to 1e-5) is therefore held to the gradient tolerance only when no weight lies between
+# the two centroid sets; the backward itself is always held to it at common centroids (the oracle's, rounded to
+# fp32 and handed to the library as C0 with the loop switched off).
+TOL_GRAD_KINK = 3e-2
+
+
+def check_workload(wl, modes=("implicit", "jfb"), alpha=1.0, want_A=False):
+    ctx = None
+    for mode in modes:
+        ref = oracle_run(wl, mode=mode, alpha=alpha, want_A=want_A)
+        out = gpu_run(wl, mode=mode, alpha=alpha, want_A=want_A, ctx=ctx)
+        ctx = out["ctx"]
+        info = out["info"][0]
+        assert info.status == 0, info
+        assert info.fwd_iters == wl.max_iter
+        assert info.adj_iters == (wl.adj_max_iter if mode == "implicit" else 0)
+        assert_close(out["C"], ref["C"], TOL_C, f"{wl.name} C")
+        assert_close(out["Wq"], ref["Wq"], TOL_C, f"{wl.name} Wq")
+        nx = kink_crossings(wl.W, out["C"], ref["C"])
+        assert_grad_close(out["dC"], ref["dC"], f"{wl.name} dC[{mode}]", nx, TOL_GRAD, TOL_GRAD_KINK)
+        assert_grad_close(out["dW"], ref["dW"], f"{wl.name} dW[{mode}]", nx, TOL_GRAD, TOL_GRAD_KINK)
+        if want_A:
+            assert np.abs(out["A"] - ref["A"]).max() <= 2e-6, "A"
+            np.testing.assert_allclose(out["A"].sum(1), 1.0, atol=2e-6)
+        # backward proper, at common centroids
+        wc = at_centroids(wl, ref["C"])
+        refc = oracle_backward_at(wc, wc.C0, mode=mode, alpha=alpha)
+        outc = gpu_run(wc, mode=mode, alpha=alpha, ctx=ctx)
+        assert np.array_equal(outc["C"], wc.C0)
+        assert_close(outc["Wq"], refc["Wq"], TOL_C, f"{wl.name} Wq at common C")
+        assert_close(outc["dC"], refc["dC"], TOL_GRAD, f"{wl.name} dC[{mode}] at common C")
+        assert_close(outc["dW"], refc["dW"], TOL_GRAD, f"{wl.name} dW[{mode}] at common C")
+
+
+# sizes span one tile, several tiles and a ragged tail for every kernel layout (k picks the layout)
+SMALL = [
+    (1, 1, 1), (2, 1, 2), (31, 1, 3), (33, 1, 4), (4095, 1, 8), (4097, 1, 16), (20001, 1, 4),
+    (7, 2, 2), (1000, 2, 4), (5003, 2, 8), (4099, 2, 16), (3001, 2, 32),
+    (5, 4, 4), (2049, 4, 8), (3000, 4, 16), (2500, 4, 17), (2051, 4, 64), (1500, 4, 100), (4100, 4, 256),
+    (3000, 1, 256), (3000, 2, 128), (2000, 1, 64),
+]
+
+
+@pytest.mark.parametrize("m,d,k", SMALL)
+def test_small_cases_fixed_iterations(m, d, k):
+    tau = {1: 0.01, 2: 0.012, 4: 0.015}[d]
+    wl = WL.single_layer(m, d, min(k, m), tau, std=0.03, seed=m + 7 * d + k, max_iter=12, adj_max_iter=8,
+                         init="rows", g_std=0.5)
+    check_workload(wl, want_A=(m <= 5003))
+
+
+def test_config1():
+    check_workload(WL.config1())
+
+
+def test_config1_paper_alpha():
+    # the paper's averaged iteration, alpha = 0.25
+    check_workload(WL.config1(), modes=("implicit",), alpha=0.25)
+
+
+def test_config2_fixed_count():
+    wl = WL.config2()
+    wl.max_iter, wl.adj_max_iter = 60, 60
+    check_workload(wl)
+
+
+def test_config2_tolerance_mode():
+    """tol 1e-6: the device decides convergence; iteration counts may differ from the oracle's by the
+    fp32 rounding of the residual, the result must be a fixed point to tol and agree to 10 tol."""
+    wl = WL.config2()
+    ref = oracle_run(wl, fixed=False)
+    out = gpu_run(wl, fixed=False)
+    info = out["info"][0]
+    assert abs(info.fwd_iters - ref["iters"]) <= 2, (info, ref["iters"])
+    assert info.fwd_residual < wl.tol
+    assert abs(info.adj_iters - ref["adj_iters"]) <= 2, (info, ref["adj_iters"])
+    if ref["adj_iters"] < wl.adj_max_iter:
+        assert info.status == 0 and info.adj_residual < wl.adj_tol
+    else:   # the adjoint hits its cap in the oracle too: advisory status, same residual
+        assert info.status == 1 and abs(info.adj_residual - ref["adj_res"]) < 0.05 * ref["adj_res"]
+    rm, _ = rel_err(out["C"], ref["C"])
+    assert rm < 2e-5
+    from oracle import idkm_ref as R
+    Cn, _, _ = R.step(wl.W.astype(np.float64), out["C"].astype(np.float64), wl.tau)
+    assert np.linalg.norm(Cn - out["C"]) / np.linalg.norm(Cn) < 2 * wl.tol
+    assert rel_err(out["dW"], ref["dW"])[0] < 1e-3
+
+
+def test_config3_batched_full():
+    wl = WL.config3()
+    gpu = gpu_run(wl, mode="implicit")
+    gpu_j = gpu_run(wl, mode="jfb", ctx=gpu["ctx"])
+    k = wl.k
+    layers = WL.split_layers(wl)
+    refs = []
+    for l, lw in enumerate(layers):
+        a, b = int(wl.layer_offsets[l]), int(wl.layer_offsets[l + 1])
+        ref = oracle_run(lw, mode="implicit")
+        refs.append(ref)
+        info = gpu["info"][l]
+        assert info.status == 0 and info.fwd_iters == wl.max_iter and info.adj_iters == wl.adj_max_iter
+        assert_close(gpu["C"][l * k:(l + 1) * k], ref["C"], TOL_C, f"layer {l} C")
+        assert_close(gpu["Wq"][a:b], ref["Wq"], TOL_C, f"layer {l} Wq")
+        nx = kink_crossings(lw.W, gpu["C"][l * k:(l + 1) * k], ref["C"])
+        assert_grad_close(gpu["dC"][l * k:(l + 1) * k], ref["dC"], f"layer {l} dC", nx, TOL_GRAD, TOL_GRAD_KINK)
+        assert_grad_close(gpu["dW"][a:b], ref["dW"], f"layer {l} dW", nx, TOL_GRAD, TOL_GRAD_KINK)
+        refj = oracle_run(lw, mode="jfb")
+        assert_grad_close(gpu_j["dC"][l * k:(l + 1) * k], refj["dC"], f"layer {l} dC jfb", nx, TOL_GRAD, TOL_GRAD_KINK)
+        assert_grad_close(gpu_j["dW"][a:b], refj["dW"], f"layer {l} dW jfb", nx, TOL_GRAD, TOL_GRAD_KINK)
+    # the whole output tensors of the batched call, in the spec norm
+    assert_close(gpu["C"], np.concatenate([r["C"] for r in refs]), TOL_C, "C, all layers")
+    assert_close(gpu["Wq"], np.concatenate([r["Wq"] for r in refs]), TOL_C, "Wq, all layers")
+    # backward proper at common centroids, all layers in one batched call
+    wc = at_centroids(wl, np.concatenate([r["C"] for r in refs]))
+    gc = gpu_run(wc, mode="implicit", ctx=gpu["ctx"])
+    gcj = gpu_run(wc, mode="jfb", ctx=gpu["ctx"])
+    for l, lw in enumerate(WL.split_layers(wc)):
+        a, b = int(wl.layer_offsets[l]), int(wl.layer_offsets[l + 1])
+        rc = oracle_backward_at(lw, lw.C0, mode="implicit")
+        assert_close(gc["dC"][l * k:(l + 1) * k], rc["dC"], TOL_GRAD, f"layer {l} dC at common C")
+        assert_close(gc["dW"][a:b], rc["dW"], TOL_GRAD, f"layer {l} dW at common C")
+        rj = oracle_backward_at(lw, lw.C0, mode="jfb")
+        assert_close(gcj["dC"][l * k:(l + 1) * k], rj["dC"], TOL_GRAD, f"layer {l} dC jfb at common C")
+        assert_close(gcj["dW"][a:b], rj["dW"], TOL_GRAD, f"layer {l} dW jfb at common C")
+
+
+def test_batched_small_layers():
+    """A batched call gives each layer the result of its own single-layer call (same tiles per layer)."""
+    shapes = [(16, 3, 3, 3), (8, 16, 1, 1), (32, 16, 3, 3), (10, 32, 1, 1)]
+    wl = WL.config3(shapes=shapes, iters=15)
+    out = gpu_run(wl)
+    for l, lw in enumerate(WL.split_layers(wl)):
+        ref = oracle_run(lw)
+        assert_close(out["C"][l * wl.k:(l + 1) * wl.k], ref["C"], TOL_C, f"layer {l}")
+        a, b = int(wl.layer_offsets[l]), int(wl.layer_offsets[l + 1])
+        nx = kink_crossings(lw.W, out["C"][l * wl.k:(l + 1) * wl.k], ref["C"])
+        assert_grad_close(out["dW"][a:b], ref["dW"], f"layer {l} dW", nx, TOL_GRAD, TOL_GRAD_KINK)
+
+
+def test_batched_unaligned_layer_offsets():
+    """Layer sizes that are not multiples of 4 force the scalar load path for d = 1."""
+    rng = np.random.default_rng(0)
+    sizes = [1001, 37, 2050, 3]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    W = (rng.standard_normal((offs[-1], 1)) * 0.05).astype(np.float32)
+    k = 3
+    C0 = np.concatenate([WL.quantile_centroids(W[offs[l]:offs[l + 1]], k) for l in range(4)])
+    G = rng.standard_normal(W.shape).astype(np.float32)
+    wl = WL.Workload("unaligned", W, C0, G, 1, k, float(np.float32(0.02)), 0.0, 10, 0.0, 6, offs, 0)
+    out = gpu_run(wl)
+    for l, lw in enumerate(WL.split_layers(wl)):
+        ref = oracle_run(lw)
+        assert_close(out["C"][l * k:(l + 1) * k], ref["C"], TOL_C, f"layer {l} C")
+        assert_close(out["Wq"][offs[l]:offs[l + 1]], ref["Wq"], TOL_C, f"layer {l} Wq")
+        nx = kink_crossings(lw.W, out["C"][l * k:(l + 1) * k], ref["C"])
+        assert_grad_close(out["dW"][offs[l]:offs[l + 1]], ref["dW"], f"layer {l} dW", nx, TOL_GRAD, TOL_GRAD_KINK)
+
+
+def test_config4_reduced_m_full_k():
+    wl = WL.config4(m=1 << 15, iters=20)
+    check_workload(wl)
+
+
+def test_run_to_run_bitwise_determinism():
+    wl = WL.config4(m=30011, k=64, iters=6)
+    a = gpu_run(wl)
+    b = gpu_run(wl)
+    for key in ("C", "Wq", "dW", "dC"):
+        assert np.array_equal(a[key], b[key]), key
+
+
+def test_zero_iterations_and_weight_on_centroid():
+    """max_iter = 0 returns C0; C0 rows are rows of W, so D_ij = 0 occurs: the sub-gradient n = 0 is used."""
+    wl = WL.single_layer(3000, 4, 16, 0.02, std=0.03, seed=5, max_iter=0, adj_max_iter=5, init="rows")
+    ref = oracle_run(wl)
+    out = gpu_run(wl)
+    assert np.array_equal(out["C"], wl.C0)
+    assert_close(out["Wq"], ref["Wq"], TOL_C, "Wq")
+    assert_close(out["dW"], ref["dW"], TOL_GRAD, "dW")
+    wl1 = WL.single_layer(3000, 1, 4, 0.02, std=0.03, seed=5, max_iter=0, adj_max_iter=5, init="rows")
+    assert_close(gpu_run(wl1)["dW"], oracle_run(wl1)["dW"], TOL_GRAD, "dW d=1")
+
+
+def test_dead_cluster_keeps_centroid():
+    wl = WL.single_layer(2000, 1, 4, 0.001, std=0.02, seed=9, max_iter=3, adj_max_iter=2)
+    wl.C0 = wl.C0.copy()
+    wl.C0[3, 0] = 1.0e4       # exp(-1e4/1e-3) underflows in fp32 and fp64 alike
+    ref = oracle_run(wl)
+    out = gpu_run(wl)
+    assert ref["dead"] == 1 and out["info"][0].dead_clusters == 1
+    assert out["C"][3, 0] == np.float32(1.0e4)
+    assert_close(out["C"][:3], ref["C"][:3], TOL_C, "C")
+    assert np.all(np.isfinite(out["dW"])) and np.all(np.isfinite(out["dC"]))
+    assert_close(out["dW"], ref["dW"], TOL_GRAD, "dW")
+
+
+def test_nonfinite_input_is_reported():
+    wl = WL.single_layer(1000, 1, 4, 0.02, seed=1, max_iter=4)
+    wl.W = wl.W.copy()
+    wl.W[17, 0] = np.nan
+    out = gpu_run(wl)
+    assert out["info"][0].status == -9
