@@ -176,6 +176,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=1 << 19)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--iters", type=int, default=0, help="override the forward and adjoint iteration counts "
+                    "(short runs for profiler captures; the reported value is then not the configured workload's)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3 if args.impl == "ours" else args.warmup
@@ -198,6 +200,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     wl = make_workload(args.workload)
+    if args.iters > 0:
+        wl.max_iter = wl.adj_max_iter = args.iters
     m, d, k, L = wl.m, wl.d, wl.k, wl.n_layers
     offs = [int(x) for x in wl.layer_offsets]
     T_f, T_a = wl.max_iter, wl.adj_max_iter

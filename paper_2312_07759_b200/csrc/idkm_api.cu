@@ -4,6 +4,7 @@
 #include "idkm_kernels.cuh"
 
 #include <math.h>
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -64,7 +65,31 @@ const KernelEntry* kernel_entry(int mode, int d, int family) {
   return nullptr;
 }
 
+// Tuning override for experiments: IDKM_FORCE_FAMILY="<mode>:<family>[,<mode>:<family>...]" forces the codebook
+// layout of a pass (used only if that layout can hold k centroids).
+static int forced_family(int mode) {
+  static int table[N_MODES];
+  static bool parsed = false;
+  if (!parsed) {
+    for (int i = 0; i < N_MODES; ++i) table[i] = -1;
+    const char* e = getenv("IDKM_FORCE_FAMILY");
+    while (e && *e) {
+      int m = -1, f = -1;
+      if (sscanf(e, "%d:%d", &m, &f) == 2 && m >= 0 && m < N_MODES && f >= 0 && f < N_FAMILY) table[m] = f;
+      e = strchr(e, ',');
+      if (e) ++e;
+    }
+    parsed = true;
+  }
+  return table[mode];
+}
+
 int pick_family(int mode, int d, int k) {
+  const int forced = forced_family(mode);
+  if (forced >= 0) {
+    const KernelEntry* e = kernel_entry(mode, d, forced);
+    if (e && e->kpl * e->lpw >= k) return forced;
+  }
   for (int f = 0; f < N_FAMILY; ++f) {
     const KernelEntry* e = kernel_entry(mode, d, f);
     if (e && e->kpl * e->lpw >= k) return f;

@@ -31,7 +31,7 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
   {                                                                                               \
     IDKM_PRECISE_ENTRY(D, 2, 1), IDKM_PRECISE_ENTRY(D, 4, 1), IDKM_PRECISE_ENTRY(D, 8, 1),        \
         IDKM_PRECISE_ENTRY(D, 8, 2), IDKM_PRECISE_ENTRY(D, 8, 4), IDKM_PRECISE_ENTRY(D, 8, 8),    \
-        IDKM_PRECISE_ENTRY(D, 8, 16), IDKM_PRECISE_ENTRY(D, 8, 32)                                \
+        IDKM_PRECISE_ENTRY(D, 8, 16), IDKM_PRECISE_ENTRY(D, 8, 32), IDKM_PRECISE_ENTRY(D, 8, 32)  \
   }
 
 // forward passes keep 16 centroids per lane, backward passes 8 (they also hold F_j and u_j/S_j)
@@ -39,13 +39,13 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
   {                                                                                               \
     IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
         IDKM_ENTRY(MODE, D, 16, 1), IDKM_ENTRY(MODE, D, 16, 2), IDKM_ENTRY(MODE, D, 16, 4),       \
-        IDKM_ENTRY(MODE, D, 16, 8), IDKM_ENTRY(MODE, D, 16, 16)                                   \
+        IDKM_ENTRY(MODE, D, 16, 8), IDKM_ENTRY(MODE, D, 16, 16), IDKM_ENTRY(MODE, D, 8, 32)       \
   }
 #define IDKM_BWD_ROW(MODE, D)                                                                     \
   {                                                                                               \
     IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
         IDKM_ENTRY(MODE, D, 8, 2), IDKM_ENTRY(MODE, D, 8, 4), IDKM_ENTRY(MODE, D, 8, 8),          \
-        IDKM_ENTRY(MODE, D, 8, 16), IDKM_ENTRY(MODE, D, 8, 32)                                    \
+        IDKM_ENTRY(MODE, D, 8, 16), IDKM_ENTRY(MODE, D, 8, 32), IDKM_ENTRY(MODE, D, 8, 32)        \
   }
 
 }  // namespace idkm

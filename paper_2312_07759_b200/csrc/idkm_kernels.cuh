@@ -94,8 +94,11 @@ struct PassCfg {
   static constexpr int GROUPS = BLOCK / LPW;
   static constexpr int VEC = (LPW == 1) ? 4 / D : 1;              // weight-vectors per 128-bit load
   static constexpr int UNROLL = (LPW == 1) ? ((KPL * D >= 32) ? 1 : 2) : 1;
-  static constexpr int WPG = (LPW == 1) ? VEC * UNROLL : 16;      // weight-vectors per group per tile
+  // weight-vectors per group per tile (bounded so that the staging buffers stay a few KB)
+  static constexpr int WPG = (LPW == 1) ? VEC * UNROLL : (LPW >= 16 ? 16 : (LPW == 8 ? 8 : 4));
   static constexpr int TILE = GROUPS * WPG;
+  // resident blocks per SM the register budget is sized for (the 32-lane layouts hold 8 centroids per lane)
+  static constexpr int MIN_BLOCKS = (LPW == 32) ? 2 : 1;
 };
 
 // ---- special-function-unit wrappers ------------------------------------------------------------
@@ -126,11 +129,18 @@ __device__ __forceinline__ float group_sum(float v) {
   for (int o = LPW / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
+// Minimum over the lanes of a group of a NON-NEGATIVE float.  Non-negative IEEE floats order like their bit
+// patterns read as unsigned integers, so a full warp does it with one integer warp-reduce instruction; with
+// sub-warp masks that instruction measured slower than the shuffles, so smaller groups shuffle.
 template <int LPW>
 __device__ __forceinline__ float group_min(float v) {
+  if constexpr (LPW == 32) {
+    return __uint_as_float(__reduce_min_sync(0xffffffffu, __float_as_uint(v)));
+  } else {
 #pragma unroll
-  for (int o = LPW / 2; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
+    for (int o = LPW / 2; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+  }
 }
 
 // block that owns tile t when n_tiles are dealt contiguously to n_blocks blocks:
@@ -340,9 +350,9 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
 
 // ---- the pass ------------------------------------------------------------------------------------
 template <int MODE, int D, int KPL, int LPW>
-__global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassParams p) {
+__global__ void __launch_bounds__(BLOCK, PassCfg<MODE, D, KPL, LPW>::MIN_BLOCKS)
+idkm_pass(const __grid_constant__ PassParams p) {
   using Cfg = PassCfg<MODE, D, KPL, LPW>;
-  constexpr int KP = Cfg::KP;
   constexpr int NACC = Cfg::NACC;
   constexpr int PLEN = Cfg::PLEN;
   constexpr int WPG = Cfg::WPG;
@@ -353,6 +363,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
   constexpr bool NEED_U = (MODE == ADJ || MODE == SCATTER);
   constexpr bool ACCUM = (NACC > 0);
   constexpr int NA = ACCUM ? NACC : 1;
+  constexpr int KH = KPL / 2;
 
   // shared: cross-warp reduction buffer (floats), reused by the last block as fp64 scratch
   constexpr int RED_BYTES = ACCUM ? NWARP * PLEN * 4 : 16;
@@ -360,6 +371,12 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
   constexpr int SMEM_BYTES = RED_BYTES > LAST_BYTES ? RED_BYTES : LAST_BYTES;
   __shared__ __align__(16) unsigned char smem_raw[SMEM_BYTES];
   __shared__ int s_flag;
+  // group-per-weight layouts stage each tile's rows in shared memory (one slot per group)
+  constexpr int STAGE = (LPW > 1) ? Cfg::GROUPS * WPG * D : 4;
+  constexpr int LD = (LPW > 1) ? (WPG + LPW - 1) / LPW : 1;   // rows each lane fetches per tile
+  __shared__ __align__(16) float wstage[STAGE];
+  __shared__ __align__(16) float gstage[NEED_G ? STAGE : 4];
+  (void)wstage; (void)gstage;
 
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -373,11 +390,16 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
   const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
   if (t_lo >= t_hi) return;
 
-  float c[KPL][D];                 // owned centroids
-  float fj[NEED_U ? KPL : 1][D];   // F(C_T, W)_j
+  // Centroids and sums are held as float2 pairs of neighbouring centroids (2h, 2h+1) so that the forward passes
+  // can use the packed fp32x2 instructions of sm_100 (one issue slot for two FMAs); c_(t, a) / acc_(t, a) give
+  // the scalar view, which resolves to a register half once the loops are unrolled.
+  float2 c2[KH][D];                // owned centroids
   float us[NEED_U ? KPL : 1][D];   // u_j / S_j (0 for a dead cluster)
-  float acc[ACCUM ? KPL : 1][NA];
-  (void)fj; (void)us; (void)acc;
+  float kap[NEED_U ? KPL : 1];     // (u_j / S_j) . F(C_T, W)_j, so that p_ij = (u_j / S_j) . w_i - kap_j
+  float2 acc2[ACCUM ? KH : 1][NA];
+  (void)kap; (void)us; (void)acc2;
+  auto c_ = [&](int t, int a) -> float& { return (t & 1) ? c2[t >> 1][a].y : c2[t >> 1][a].x; };
+  auto acc_ = [&](int t, int a) -> float& { return (t & 1) ? acc2[t >> 1][a].y : acc2[t >> 1][a].x; };
 
   int layer = 0;
   while (p.lt.tile_off[layer + 1] <= t_lo) ++layer;
@@ -390,19 +412,22 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
     for (int t = 0; t < KPL; ++t) {
       const int j = gl * KPL + t;
 #pragma unroll
-      for (int a = 0; a < D; ++a) c[t][a] = (j < k) ? Cl[j * D + a] : PAD_COORD;
+      for (int a = 0; a < D; ++a) c_(t, a) = (j < k) ? Cl[j * D + a] : PAD_COORD;
       if constexpr (NEED_U) {
         const float s = (j < k) ? p.S[(size_t)l * k + j] : 0.f;
         const float inv = (s >= S_MIN_F) ? 1.f / s : 0.f;
+        float kp = 0.f;
 #pragma unroll
         for (int a = 0; a < D; ++a) {
-          fj[t][a] = (j < k) ? p.F[((size_t)l * k + j) * D + a] : 0.f;
+          const float f = (j < k) ? p.F[((size_t)l * k + j) * D + a] : 0.f;
           us[t][a] = (j < k) ? p.u[((size_t)l * k + j) * D + a] * inv : 0.f;
+          kp = fmaf(us[t][a], f, kp);
         }
+        kap[t] = kp;
       }
       if constexpr (ACCUM) {
 #pragma unroll
-        for (int a = 0; a < NA; ++a) acc[t][a] = 0.f;
+        for (int a = 0; a < NA; ++a) acc_(t, a) = 0.f;
       }
     }
   };
@@ -411,49 +436,93 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
   auto process = [&](const float (&w)[D], const float (&gi)[D], bool valid, long long row, float (&out)[D]) {
     float dist[KPL];
     float rs[(D > 1 && !FWD) ? KPL : 1];
-    (void)rs;
+    (void)rs; (void)dist;
+    float e[KPL];
     float lmin = 3.0e38f;
+    float lsum = 0.f;
+    float gsum, r;
+    if constexpr (FWD && D > 1) {
+      // packed path: two centroids per instruction
+      const float2 neg1 = make_float2(-1.f, -1.f);
+      float2 d2[KH];
 #pragma unroll
-    for (int t = 0; t < KPL; ++t) {
-      if constexpr (D == 1) {
-        dist[t] = fabsf(w[0] - c[t][0]);
-      } else {
-        float sq = 0.f;
+      for (int h = 0; h < KH; ++h) {
+        float2 sq = make_float2(0.f, 0.f);
 #pragma unroll
         for (int a = 0; a < D; ++a) {
-          const float df = w[a] - c[t][a];
-          sq = fmaf(df, df, sq);
+          const float2 df = __ffma2_rn(c2[h][a], neg1, make_float2(w[a], w[a]));   // w - c, exactly as a subtraction
+          sq = (a == 0) ? __fmul2_rn(df, df) : __ffma2_rn(df, df, sq);
         }
-        if constexpr (FWD) {
-          dist[t] = sqrt_approx(sq);
-        } else {
-          rs[t] = rsqrt_approx(fmaxf(sq, 1e-30f));
-          dist[t] = sq * rs[t];
-        }
+        d2[h] = make_float2(sqrt_approx(sq.x), sqrt_approx(sq.y));
+        lmin = fminf(lmin, fminf(d2[h].x, d2[h].y));
       }
-      lmin = fminf(lmin, dist[t]);
-    }
-    const float gmin = group_min<LPW>(lmin);
-    const float mref = gmin * p.scale;
-    float e[KPL];
-    float lsum = 0.f;
+      const float gmin = group_min<LPW>(lmin);
+      const float mref = gmin * p.scale;
+      const float2 nscale = make_float2(-p.scale, -p.scale), mref2 = make_float2(mref, mref);
+      float2 ls2 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int t = 0; t < KPL; ++t) {
-      e[t] = ex2_approx(fmaf(-p.scale, dist[t], mref));
-      lsum += e[t];
+      for (int h = 0; h < KH; ++h) {
+        const float2 x = __ffma2_rn(d2[h], nscale, mref2);
+        const float2 ee = make_float2(ex2_approx(x.x), ex2_approx(x.y));
+        e[2 * h] = ee.x;
+        e[2 * h + 1] = ee.y;
+        ls2 = __fadd2_rn(ls2, ee);
+      }
+      lsum = ls2.x + ls2.y;
+      gsum = group_sum<LPW>(lsum);
+      r = valid ? rcp_approx(gsum) : 0.f;
+    } else {
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        if constexpr (D == 1) {
+          dist[t] = fabsf(w[0] - c_(t, 0));
+        } else {
+          float sq = 0.f;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const float df = w[a] - c_(t, a);
+            sq = fmaf(df, df, sq);
+          }
+          if constexpr (FWD) {
+            dist[t] = sqrt_approx(sq);
+          } else {
+            rs[t] = rsqrt_approx(fmaxf(sq, 1e-30f));
+            dist[t] = sq * rs[t];
+          }
+        }
+        lmin = fminf(lmin, dist[t]);
+      }
+      const float gmin = group_min<LPW>(lmin);
+      const float mref = gmin * p.scale;
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        e[t] = ex2_approx(fmaf(-p.scale, dist[t], mref));
+        lsum += e[t];
+      }
+      gsum = group_sum<LPW>(lsum);
+      r = valid ? rcp_approx(gsum) : 0.f;
     }
-    const float gsum = group_sum<LPW>(lsum);
-    const float r = valid ? rcp_approx(gsum) : 0.f;
 
     if constexpr (MODE == STEP || MODE == FINAL) {
       float rw[D];
 #pragma unroll
       for (int a = 0; a < D; ++a) rw[a] = r * w[a];
+      if constexpr (D > 1) {
+        const float2 r2 = make_float2(r, r);
 #pragma unroll
-      for (int t = 0; t < KPL; ++t) {
-        acc[t][0] = fmaf(e[t], r, acc[t][0]);
+        for (int h = 0; h < KH; ++h) {
+          const float2 ee = make_float2(e[2 * h], e[2 * h + 1]);
+          acc2[h][0] = __ffma2_rn(ee, r2, acc2[h][0]);
 #pragma unroll
-        for (int a = 0; a < D; ++a) acc[t][1 + a] = fmaf(e[t], rw[a], acc[t][1 + a]);
+          for (int a = 0; a < D; ++a) acc2[h][1 + a] = __ffma2_rn(ee, make_float2(rw[a], rw[a]), acc2[h][1 + a]);
+        }
+      } else {
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          acc_(t, 0) = fmaf(e[t], r, acc_(t, 0));
+#pragma unroll
+          for (int a = 0; a < D; ++a) acc_(t, 1 + a) = fmaf(e[t], rw[a], acc_(t, 1 + a));
+        }
       }
       if constexpr (MODE == FINAL) {
         if (p.Wq != nullptr) {
@@ -461,7 +530,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
           for (int a = 0; a < D; ++a) {
             float s = 0.f;
 #pragma unroll
-            for (int t = 0; t < KPL; ++t) s = fmaf(e[t], (gl * KPL + t < k) ? c[t][a] : 0.f, s);
+            for (int t = 0; t < KPL; ++t) s = fmaf(e[t], (gl * KPL + t < k) ? c_(t, a) : 0.f, s);
             out[a] = group_sum<LPW>(s) * r;
           }
         }
@@ -481,13 +550,14 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
         float v = 0.f;
+        if constexpr (NEED_U) {
+          v = -kap[t];
+#pragma unroll
+          for (int a = 0; a < D; ++a) v = fmaf(us[t][a], w[a], v);
+        }
         if constexpr (NEED_G) {
 #pragma unroll
-          for (int a = 0; a < D; ++a) v = fmaf(gi[a], (gl * KPL + t < k) ? c[t][a] : 0.f, v);
-        }
-        if constexpr (NEED_U) {
-#pragma unroll
-          for (int a = 0; a < D; ++a) v = fmaf(us[t][a], w[a] - fj[t][a], v);
+          for (int a = 0; a < D; ++a) v = fmaf(gi[a], (gl * KPL + t < k) ? c_(t, a) : 0.f, v);
         }
         z[t] = v;
         lz = fmaf(e[t], v, lz);
@@ -500,15 +570,16 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
         const float at = e[t] * r;                    // A_ij
-        const float et = e[t] * rt * (z[t] - zbar);   // e_ij(z) / tau
+        float et = e[t] * rt * (z[t] - zbar);         // e_ij(z) / tau
+        if constexpr (D > 1) et *= rs[t];             // ... / D_ij, so that et * (w - c) = e_ij(z) n_ij / tau
 #pragma unroll
         for (int a = 0; a < D; ++a) {
-          const float df = w[a] - c[t][a];
+          const float df = w[a] - c_(t, a);
           float n;
           if constexpr (D == 1) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
-          else n = df * rs[t];
-          if constexpr (MODE == GRAD) acc[t][a] = fmaf(at, gi[a], fmaf(et, n, acc[t][a]));
-          if constexpr (MODE == ADJ) acc[t][a] = fmaf(et, n, acc[t][a]);
+          else n = df;
+          if constexpr (MODE == GRAD) acc_(t, a) = fmaf(at, gi[a], fmaf(et, n, acc_(t, a)));
+          if constexpr (MODE == ADJ) acc_(t, a) = fmaf(et, n, acc_(t, a));
           if constexpr (MODE == SCATTER) dwl[a] = fmaf(at, us[t][a], fmaf(-et, n, dwl[a]));
         }
       }
@@ -530,17 +601,17 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
       for (int t = 0; t < KPL; ++t)
 #pragma unroll
         for (int a = 0; a < NA; ++a) {
-          float v = acc[t][a];
+          float v = acc_(t, a);
 #pragma unroll
           for (int o = LPW; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-          acc[t][a] = v;
+          acc_(t, a) = v;
         }
       __syncthreads();
       if (lane < LPW) {
 #pragma unroll
         for (int t = 0; t < KPL; ++t)
 #pragma unroll
-          for (int a = 0; a < NA; ++a) red[warp * PLEN + (gl * KPL + t) * NA + a] = acc[t][a];
+          for (int a = 0; a < NA; ++a) red[warp * PLEN + (gl * KPL + t) * NA + a] = acc_(t, a);
       }
       __syncthreads();
       const int slot = b + l;
@@ -555,6 +626,46 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
     }
   };
 
+  // rows fetched one tile ahead by this lane (group-per-weight layouts)
+  float pw[LD][D], pg[NEED_G ? LD : 1][D];
+  (void)pw; (void)pg;
+  auto fetch = [&](int tl, int ly) {
+    if constexpr (LPW > 1) {
+      const long long r0 = p.lt.row_off[ly];
+      const long long rws = p.lt.row_off[ly + 1] - r0;
+      const long long gb = (long long)(tl - p.lt.tile_off[ly]) * TILE + (long long)grp * WPG;
+#pragma unroll
+      for (int q = 0; q < LD; ++q) {
+        const int idx = gl + q * LPW;
+        if (idx < WPG) {
+          const long long loc = gb + idx;
+          const long long grow = r0 + ((loc < rws) ? loc : 0);
+          if constexpr (D == 4) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(p.W + grow * 4));
+            pw[q][0] = x.x; pw[q][1] = x.y; pw[q][2] = x.z; pw[q][3] = x.w;
+          } else if constexpr (D == 2) {
+            const float2 x = __ldg(reinterpret_cast<const float2*>(p.W + grow * 2));
+            pw[q][0] = x.x; pw[q][1] = x.y;
+          } else {
+            pw[q][0] = __ldg(p.W + grow);
+          }
+          if constexpr (NEED_G) {
+            if constexpr (D == 4) {
+              const float4 y = __ldg(reinterpret_cast<const float4*>(p.G + grow * 4));
+              pg[q][0] = y.x; pg[q][1] = y.y; pg[q][2] = y.z; pg[q][3] = y.w;
+            } else if constexpr (D == 2) {
+              const float2 y = __ldg(reinterpret_cast<const float2*>(p.G + grow * 2));
+              pg[q][0] = y.x; pg[q][1] = y.y;
+            } else {
+              pg[q][0] = __ldg(p.G + grow);
+            }
+          }
+        }
+      }
+    }
+  };
+  fetch(t_lo, layer);
+
   // ---- persistent loop over this block's tiles -------------------------------------------------
   for (int tile = t_lo; tile < t_hi; ++tile) {
     while (p.lt.tile_off[layer + 1] <= tile) ++layer;
@@ -566,6 +677,27 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
       else if constexpr (MODE == ADJ) layer_active = (p.st[layer].adj_done == 0);
       else layer_active = true;
       if (layer_active) load_layer(layer);
+    }
+    if constexpr (LPW > 1) {
+      // park the rows fetched for this tile, then fetch the next tile's while this one is processed
+      __syncwarp();
+#pragma unroll
+      for (int q = 0; q < LD; ++q) {
+        const int idx = gl + q * LPW;
+        if (idx < WPG) {
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            wstage[(grp * WPG + idx) * D + a] = pw[q][a];
+            if constexpr (NEED_G) gstage[(grp * WPG + idx) * D + a] = pg[q][a];
+          }
+        }
+      }
+      __syncwarp();
+      if (tile + 1 < t_hi) {
+        int ly2 = layer;
+        while (p.lt.tile_off[ly2 + 1] <= tile + 1) ++ly2;
+        fetch(tile + 1, ly2);
+      }
     }
     if (!layer_active) continue;
     const long long row0 = p.lt.row_off[layer];
@@ -646,7 +778,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
         }
       }
     } else {
-      // group-per-weight: every lane of the group reads the same row (one broadcast request)
+      // group-per-weight: the group reads one staged row at a time (a shared-memory broadcast)
       const long long gbase = tbase + (long long)grp * WPG;
 #pragma unroll 2
       for (int t = 0; t < WPG; ++t) {
@@ -654,26 +786,28 @@ __global__ void __launch_bounds__(BLOCK) idkm_pass(const __grid_constant__ PassP
         const bool ok = (loc < rows);
         const long long grow = row0 + (ok ? loc : 0);
         float w[D], gi[D], outv[D];
+        const float* ws = wstage + (grp * WPG + t) * D;
         if constexpr (D == 4) {
-          const float4 x = __ldg(reinterpret_cast<const float4*>(p.W + grow * 4));
+          const float4 x = *reinterpret_cast<const float4*>(ws);
           w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
         } else if constexpr (D == 2) {
-          const float2 x = __ldg(reinterpret_cast<const float2*>(p.W + grow * 2));
+          const float2 x = *reinterpret_cast<const float2*>(ws);
           w[0] = x.x; w[1] = x.y;
         } else {
-          w[0] = __ldg(p.W + grow);
+          w[0] = ws[0];
         }
 #pragma unroll
         for (int a = 0; a < D; ++a) gi[a] = 0.f;
         if constexpr (NEED_G) {
+          const float* gs = gstage + (grp * WPG + t) * D;
           if constexpr (D == 4) {
-            const float4 y = __ldg(reinterpret_cast<const float4*>(p.G + grow * 4));
+            const float4 y = *reinterpret_cast<const float4*>(gs);
             gi[0] = y.x; gi[1] = y.y; gi[2] = y.z; gi[3] = y.w;
           } else if constexpr (D == 2) {
-            const float2 y = __ldg(reinterpret_cast<const float2*>(p.G + grow * 2));
+            const float2 y = *reinterpret_cast<const float2*>(gs);
             gi[0] = y.x; gi[1] = y.y;
           } else {
-            gi[0] = __ldg(p.G + grow);
+            gi[0] = gs[0];
           }
         }
         process(w, gi, ok, grow, outv);
@@ -864,7 +998,7 @@ struct KernelEntry {
   int kpl, lpw, tile, plen;
 };
 // family index f: 0..7 -> supports k <= kpl*lpw
-constexpr int N_FAMILY = 8;
+constexpr int N_FAMILY = 9;
 const KernelEntry* kernel_entry(int mode, int d, int family);
 int pick_family(int mode, int d, int k);
 
