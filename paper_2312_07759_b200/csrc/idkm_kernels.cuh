@@ -123,6 +123,19 @@ __device__ __forceinline__ float rcp_approx(float x) {
   return y;
 }
 
+// Pairwise (tree) sum (OP 0) or minimum (OP 1) of a register array: log2(N) dependent steps instead of N.
+template <int N, int OP>
+__device__ __forceinline__ float tree_reduce(const float (&x)[N]) {
+  float t[N];
+#pragma unroll
+  for (int i = 0; i < N; ++i) t[i] = x[i];
+#pragma unroll
+  for (int s = 1; s < N; s <<= 1)
+#pragma unroll
+    for (int i = 0; i + s < N; i += 2 * s) t[i] = (OP == 0) ? t[i] + t[i + s] : fminf(t[i], t[i + s]);
+  return t[0];
+}
+
 template <int LPW>
 __device__ __forceinline__ float group_sum(float v) {
 #pragma unroll
@@ -390,9 +403,10 @@ idkm_pass(const __grid_constant__ PassParams p) {
   const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
   if (t_lo >= t_hi) return;
 
-  // Centroids and sums are held as float2 pairs of neighbouring centroids (2h, 2h+1) so that the forward passes
-  // can use the packed fp32x2 instructions of sm_100 (one issue slot for two FMAs); c_(t, a) / acc_(t, a) give
-  // the scalar view, which resolves to a register half once the loops are unrolled.
+  // Centroids and sums are held as float2 pairs of neighbouring centroids (2h, 2h+1); c_(t, a) / acc_(t, a) give
+  // the scalar view, which resolves to a register half once the loops are unrolled.  (The packed fp32x2
+  // instructions of sm_100 were measured on this layout: they halve the issue slots of the FMAs but run on half of
+  // the FMA pipe, and the step came out slower, so the arithmetic below is scalar.)
   float2 c2[KH][D];                // owned centroids
   float us[NEED_U ? KPL : 1][D];   // u_j / S_j (0 for a dead cluster)
   float kap[NEED_U ? KPL : 1];     // (u_j / S_j) . F(C_T, W)_j, so that p_ij = (u_j / S_j) . w_i - kap_j
@@ -441,37 +455,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
     float lmin = 3.0e38f;
     float lsum = 0.f;
     float gsum, r;
-    if constexpr (FWD && D > 1) {
-      // packed path: two centroids per instruction
-      const float2 neg1 = make_float2(-1.f, -1.f);
-      float2 d2[KH];
-#pragma unroll
-      for (int h = 0; h < KH; ++h) {
-        float2 sq = make_float2(0.f, 0.f);
-#pragma unroll
-        for (int a = 0; a < D; ++a) {
-          const float2 df = __ffma2_rn(c2[h][a], neg1, make_float2(w[a], w[a]));   // w - c, exactly as a subtraction
-          sq = (a == 0) ? __fmul2_rn(df, df) : __ffma2_rn(df, df, sq);
-        }
-        d2[h] = make_float2(sqrt_approx(sq.x), sqrt_approx(sq.y));
-        lmin = fminf(lmin, fminf(d2[h].x, d2[h].y));
-      }
-      const float gmin = group_min<LPW>(lmin);
-      const float mref = gmin * p.scale;
-      const float2 nscale = make_float2(-p.scale, -p.scale), mref2 = make_float2(mref, mref);
-      float2 ls2 = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int h = 0; h < KH; ++h) {
-        const float2 x = __ffma2_rn(d2[h], nscale, mref2);
-        const float2 ee = make_float2(ex2_approx(x.x), ex2_approx(x.y));
-        e[2 * h] = ee.x;
-        e[2 * h + 1] = ee.y;
-        ls2 = __fadd2_rn(ls2, ee);
-      }
-      lsum = ls2.x + ls2.y;
-      gsum = group_sum<LPW>(lsum);
-      r = valid ? rcp_approx(gsum) : 0.f;
-    } else {
+    {
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
         if constexpr (D == 1) {
@@ -490,15 +474,15 @@ idkm_pass(const __grid_constant__ PassParams p) {
             dist[t] = sq * rs[t];
           }
         }
-        lmin = fminf(lmin, dist[t]);
       }
+      lmin = tree_reduce<KPL, 1>(dist);
       const float gmin = group_min<LPW>(lmin);
       const float mref = gmin * p.scale;
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
         e[t] = ex2_approx(fmaf(-p.scale, dist[t], mref));
-        lsum += e[t];
       }
+      lsum = tree_reduce<KPL, 0>(e);
       gsum = group_sum<LPW>(lsum);
       r = valid ? rcp_approx(gsum) : 0.f;
     }
@@ -507,31 +491,20 @@ idkm_pass(const __grid_constant__ PassParams p) {
       float rw[D];
 #pragma unroll
       for (int a = 0; a < D; ++a) rw[a] = r * w[a];
-      if constexpr (D > 1) {
-        const float2 r2 = make_float2(r, r);
 #pragma unroll
-        for (int h = 0; h < KH; ++h) {
-          const float2 ee = make_float2(e[2 * h], e[2 * h + 1]);
-          acc2[h][0] = __ffma2_rn(ee, r2, acc2[h][0]);
+      for (int t = 0; t < KPL; ++t) {
+        acc_(t, 0) = fmaf(e[t], r, acc_(t, 0));
 #pragma unroll
-          for (int a = 0; a < D; ++a) acc2[h][1 + a] = __ffma2_rn(ee, make_float2(rw[a], rw[a]), acc2[h][1 + a]);
-        }
-      } else {
-#pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          acc_(t, 0) = fmaf(e[t], r, acc_(t, 0));
-#pragma unroll
-          for (int a = 0; a < D; ++a) acc_(t, 1 + a) = fmaf(e[t], rw[a], acc_(t, 1 + a));
-        }
+        for (int a = 0; a < D; ++a) acc_(t, 1 + a) = fmaf(e[t], rw[a], acc_(t, 1 + a));
       }
       if constexpr (MODE == FINAL) {
         if (p.Wq != nullptr) {
 #pragma unroll
           for (int a = 0; a < D; ++a) {
-            float s = 0.f;
+            float sp[2] = {0.f, 0.f};
 #pragma unroll
-            for (int t = 0; t < KPL; ++t) s = fmaf(e[t], (gl * KPL + t < k) ? c_(t, a) : 0.f, s);
-            out[a] = group_sum<LPW>(s) * r;
+            for (int t = 0; t < KPL; ++t) sp[t & 1] = fmaf(e[t], (gl * KPL + t < k) ? c_(t, a) : 0.f, sp[t & 1]);
+            out[a] = group_sum<LPW>(sp[0] + sp[1]) * r;
           }
         }
         if (p.A != nullptr && valid) {
@@ -546,7 +519,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
     } else {
       // z_ij: what the softmax Jacobian is contracted with (q for GRAD, p for ADJ, q + p for SCATTER)
       float z[KPL];
-      float lz = 0.f;
+      float lzp[4] = {0.f, 0.f, 0.f, 0.f};   // four interleaved partial sums keep the dependent chain short
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
         float v = 0.f;
@@ -560,9 +533,9 @@ idkm_pass(const __grid_constant__ PassParams p) {
           for (int a = 0; a < D; ++a) v = fmaf(gi[a], (gl * KPL + t < k) ? c_(t, a) : 0.f, v);
         }
         z[t] = v;
-        lz = fmaf(e[t], v, lz);
+        lzp[t & 3] = fmaf(e[t], v, lzp[t & 3]);
       }
-      const float zbar = group_sum<LPW>(lz) * r;
+      const float zbar = group_sum<LPW>((lzp[0] + lzp[1]) + (lzp[2] + lzp[3])) * r;
       const float rt = r * p.inv_tau;
       float dwl[D];
 #pragma unroll
