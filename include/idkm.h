@@ -53,6 +53,7 @@ extern "C" {
 #define IDKM_ERR_ORDER (-7)      /* idkm_backward without a preceding idkm_forward              */
 #define IDKM_ERR_CUDA (-8)       /* a CUDA runtime call failed                                  */
 #define IDKM_ERR_NONFINITE (-9)  /* device: NaN/Inf met in W, C or the sums                     */
+#define IDKM_ERR_NOALLOC_TOO_LARGE (-11) /* idkm_step_noalloc: the problem needs more than the built-in scratch */
 #define IDKM_ERR_DIVERGED (-10)  /* device: adjoint iteration produced non-finite values or its
                                     residual grew 10 steps running (Section 4.2: retry with a
                                     smaller alpha)                                              */
@@ -155,6 +156,34 @@ int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_
  */
 int idkm_set_timing(idkm_ctx* ctx, int enable);
 int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out);
+
+/*
+ * One application of the map, C_out = F(C_in, W), that allocates nothing.  (The paper has no
+ * counterpart: this exists for callers, not for the method.)
+ *
+ * For code that cannot obtain device memory at the point of the call: an allocator or memory-pool
+ * callback, a server that gave its whole device budget to a fixed arena at start-up, a plug-in that may
+ * not touch its host's CUDA allocator.  Such callers cannot supply the workspace the other entry points
+ * ask for.  Here the bookkeeping of the fused step (per-block partial sums and the layer's ticket and
+ * counters) lives in a fixed array of IDKM_NOALLOC_SCRATCH_BYTES inside the library image; every GPU
+ * that loads the library holds those bytes until the process exits.  The call makes no cudaMalloc,
+ * cudaFree or other allocating call and needs no idkm_ctx.
+ *
+ * W [m][d], C_in [k][d], C_out [k][d] are device pointers, 16-byte aligned, owned by the caller; C_in and
+ * C_out may alias.  The result is that of idkm_forward with max_iter = 1 (same kernels, same reduction
+ * order).  Asynchronous on cuda_stream.
+ *
+ * Limits and sharing.  Returns IDKM_ERR_NOALLOC_TOO_LARGE when (resident blocks + 1) * padded k * (d+1)
+ * * 8 bytes + 256 exceeds IDKM_NOALLOC_SCRATCH_BYTES; every supported (d, k) fits on a B200, the check
+ * guards larger parts.  All calls on a device share the one array, which still holds the previous call's
+ * contents when the next begins: the call clears what must start at zero itself, but two calls that
+ * overlap on the GPU (different streams, or different host threads) race on it -- serialise them.
+ * The first call on each device looks up the array's device address (with that device current) and the
+ * SM count; make that first call outside any stream capture.
+ */
+#define IDKM_NOALLOC_SCRATCH_BYTES (4u << 20)
+int idkm_step_noalloc(const float* W, int64_t m, int d, const float* C_in, int k, float tau, float* C_out,
+                      void* cuda_stream);
 
 /* Number of kernels this ctx has launched since idkm_create (for accounting in benchmarks). */
 int64_t idkm_launch_count(const idkm_ctx* ctx);

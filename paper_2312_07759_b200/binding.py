@@ -58,6 +58,8 @@ lib.idkm_set_timing.argtypes = [_vp, C.c_int]
 lib.idkm_set_timing.restype = C.c_int
 lib.idkm_get_phase_ms.argtypes = [_vp, C.POINTER(C.c_float)]
 lib.idkm_get_phase_ms.restype = C.c_int
+lib.idkm_step_noalloc.argtypes = [_fp, C.c_int64, C.c_int, _fp, C.c_int, C.c_float, _fp, _vp]
+lib.idkm_step_noalloc.restype = C.c_int
 lib.idkm_launch_count.argtypes = [_vp]
 lib.idkm_launch_count.restype = C.c_int64
 lib.idkm_status_string.argtypes = [C.c_int]
@@ -100,6 +102,18 @@ class ForwardResult:
     C: "object"          # torch [L*k, d]
     Wq: "object"         # torch [m, d] or None
     A: "object"          # torch [m, k] or None
+
+
+def step_noalloc(W, C_in, tau: float, C_out=None, stream=None):
+    """``idkm_step_noalloc``: C_out = F(C_in, W) on CUDA tensors without any allocation inside the library.
+    The caller passes C_out to keep the call itself allocation-free; if omitted it is created here, by torch."""
+    import torch
+    assert W.is_cuda and C_in.is_cuda and W.dtype == torch.float32 and W.is_contiguous() and C_in.is_contiguous()
+    if C_out is None:
+        C_out = torch.empty_like(C_in)
+    _check(lib.idkm_step_noalloc(_ptr(W), int(W.shape[0]), int(W.shape[1]), _ptr(C_in), int(C_in.shape[0]),
+                                 float(tau), _ptr(C_out), _stream(stream)))
+    return C_out
 
 
 class Context:

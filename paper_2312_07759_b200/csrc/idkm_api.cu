@@ -531,6 +531,7 @@ const char* idkm_status_string(int status) {
     case IDKM_ERR_CUDA: return "CUDA runtime error";
     case IDKM_ERR_NONFINITE: return "non-finite value met on the device";
     case IDKM_ERR_DIVERGED: return "adjoint iteration diverged";
+    case IDKM_ERR_NOALLOC_TOO_LARGE: return "problem needs more than the library's built-in scratch";
   }
   return "unknown status";
 }
