@@ -177,7 +177,7 @@ static int blocks_per_sm(idkm_ctx* ctx, int mode, int d, int family) {
   if (slot == 0) {
     int n = 0;
     const KernelEntry* e = kernel_entry(mode, d, family);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, e->func, BLOCK, 0) != cudaSuccess || n < 1) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, e->func, BLOCK, e->dyn_smem) != cudaSuccess || n < 1) {
       (void)cudaGetLastError();
       n = 1;
     }

@@ -7,14 +7,23 @@ namespace idkm {
 
 template <int MODE, int D, int KPL, int LPW>
 static cudaError_t launch_one(const PassParams& p, int grid, cudaStream_t stream) {
-  idkm_pass<MODE, D, KPL, LPW><<<grid, BLOCK, 0, stream>>>(p);
+  constexpr int DYN = PassCfg<MODE, D, KPL, LPW>::DYN_SMEM;
+  static bool configured = false;   // static + dynamic shared memory may exceed the 48 KB default
+  if (!configured) {
+    const cudaError_t rc = cudaFuncSetAttribute(idkm_pass<MODE, D, KPL, LPW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                DYN > 0 ? DYN : 1);
+    if (rc != cudaSuccess) return rc;
+    configured = true;
+  }
+  idkm_pass<MODE, D, KPL, LPW><<<grid, BLOCK, DYN, stream>>>(p);
   return cudaGetLastError();
 }
 
 #define IDKM_ENTRY(MODE, D, KPL, LPW)                                                             \
   {                                                                                               \
     &launch_one<MODE, D, KPL, LPW>, (const void*)&idkm_pass<MODE, D, KPL, LPW>, KPL, LPW,         \
-        PassCfg<MODE, D, KPL, LPW>::TILE, PassCfg<MODE, D, KPL, LPW>::PLEN                        \
+        PassCfg<MODE, D, KPL, LPW>::TILE, PassCfg<MODE, D, KPL, LPW>::PLEN,                       \
+        PassCfg<MODE, D, KPL, LPW>::DYN_SMEM                                                      \
   }
 
 template <int D, int KPL, int LPW>
@@ -25,7 +34,7 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
 #define IDKM_PRECISE_ENTRY(D, KPL, LPW)                                                           \
   {                                                                                               \
     &launch_precise<D, KPL, LPW>, (const void*)&idkm_step_precise<D, KPL, LPW>, KPL, LPW,         \
-        PreciseCfg<D, KPL, LPW>::TILE, PreciseCfg<D, KPL, LPW>::PLEN                              \
+        PreciseCfg<D, KPL, LPW>::TILE, PreciseCfg<D, KPL, LPW>::PLEN, 0                           \
   }
 #define IDKM_PRECISE_ROW(D)                                                                       \
   {                                                                                               \

@@ -97,6 +97,12 @@ struct PassCfg {
   // weight-vectors per group per tile (bounded so that the staging buffers stay a few KB)
   static constexpr int WPG = (LPW == 1) ? VEC * UNROLL : (LPW >= 16 ? 16 : (LPW == 8 ? 8 : 4));
   static constexpr int TILE = GROUPS * WPG;
+  // Each thread's sums are moved out of its registers into a private fp32 slot in (dynamic) shared memory every
+  // SPILL_TILES tiles, i.e. after about 64 weight-vectors.  A long-running fp32 accumulator silently drops the
+  // many terms that are smaller than half its ulp (the attention of far-away weights), a one-sided loss that was
+  // measured to grow in proportion to the number of terms; 64-term chunks keep it below 3e-8 relative.
+  static constexpr int SPILL_TILES = (64 / WPG) > 0 ? (64 / WPG) : 1;
+  static constexpr int DYN_SMEM = (NACC > 0) ? BLOCK * KPL * NACC * 4 : 0;
   // resident blocks per SM the register budget is sized for (the 32-lane layouts hold 8 centroids per lane)
   static constexpr int MIN_BLOCKS = (LPW == 32) ? 2 : 1;
 };
@@ -387,6 +393,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
   // group-per-weight layouts stage each tile's rows in shared memory (one slot per group)
   constexpr int STAGE = (LPW > 1) ? Cfg::GROUPS * WPG * D : 4;
   constexpr int LD = (LPW > 1) ? (WPG + LPW - 1) / LPW : 1;   // rows each lane fetches per tile
+  extern __shared__ __align__(16) float slots[];   // [KPL * NA][BLOCK]: second-level sums, one column per thread
   __shared__ __align__(16) float wstage[STAGE];
   __shared__ __align__(16) float gstage[NEED_G ? STAGE : 4];
   (void)wstage; (void)gstage;
@@ -441,8 +448,23 @@ idkm_pass(const __grid_constant__ PassParams p) {
       }
       if constexpr (ACCUM) {
 #pragma unroll
-        for (int a = 0; a < NA; ++a) acc_(t, a) = 0.f;
+        for (int a = 0; a < NA; ++a) {
+          acc_(t, a) = 0.f;
+          slots[(t * NA + a) * BLOCK + tid] = 0.f;
+        }
       }
+    }
+  };
+  int since_spill = 0;
+  auto spill = [&]() {
+    if constexpr (ACCUM) {
+#pragma unroll
+      for (int t = 0; t < KPL; ++t)
+#pragma unroll
+        for (int a = 0; a < NA; ++a) {
+          slots[(t * NA + a) * BLOCK + tid] += acc_(t, a);
+          acc_(t, a) = 0.f;
+        }
     }
   };
 
@@ -569,12 +591,12 @@ idkm_pass(const __grid_constant__ PassParams p) {
       return;
     } else {
       float* red = reinterpret_cast<float*>(smem_raw);
-      // across the groups of a warp (lanes with equal gl)
+      // across the groups of a warp (lanes with equal gl); the thread's own two levels are joined first
 #pragma unroll
       for (int t = 0; t < KPL; ++t)
 #pragma unroll
         for (int a = 0; a < NA; ++a) {
-          float v = acc_(t, a);
+          float v = acc_(t, a) + slots[(t * NA + a) * BLOCK + tid];
 #pragma unroll
           for (int o = LPW; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
           acc_(t, a) = v;
@@ -650,6 +672,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
       else if constexpr (MODE == ADJ) layer_active = (p.st[layer].adj_done == 0);
       else layer_active = true;
       if (layer_active) load_layer(layer);
+      since_spill = 0;
     }
     if constexpr (LPW > 1) {
       // park the rows fetched for this tile, then fetch the next tile's while this one is processed
@@ -792,6 +815,12 @@ idkm_pass(const __grid_constant__ PassParams p) {
             else dst[grow] = outv[0];
           }
         }
+      }
+    }
+    if constexpr (ACCUM) {
+      if (++since_spill == Cfg::SPILL_TILES) {
+        spill();
+        since_spill = 0;
       }
     }
   }
@@ -969,6 +998,7 @@ struct KernelEntry {
   LaunchFn launch;
   const void* func;
   int kpl, lpw, tile, plen;
+  int dyn_smem;   // dynamic shared memory the launch asks for (bytes)
 };
 // family index f: 0..7 -> supports k <= kpl*lpw
 constexpr int N_FAMILY = 9;

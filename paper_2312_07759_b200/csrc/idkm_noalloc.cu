@@ -68,7 +68,7 @@ static int noalloc_table(const KernelEntry* e, int64_t m, int sms, LayerTable* l
   }
   lt->tiles_total = (int)tiles;
   int per_sm = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, e->func, BLOCK, 0) != cudaSuccess || per_sm < 1) {
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, e->func, BLOCK, e->dyn_smem) != cudaSuccess || per_sm < 1) {
     (void)cudaGetLastError();
     per_sm = 1;
   }
