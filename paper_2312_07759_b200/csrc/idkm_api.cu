@@ -177,6 +177,8 @@ static int blocks_per_sm(idkm_ctx* ctx, int mode, int d, int family) {
   if (slot == 0) {
     int n = 0;
     const KernelEntry* e = kernel_entry(mode, d, family);
+    // static + dynamic shared memory can exceed the 48 KB default: raise the limit before asking for the occupancy
+    if (e->dyn_smem > 0) (void)cudaFuncSetAttribute(e->func, cudaFuncAttributeMaxDynamicSharedMemorySize, e->dyn_smem);
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, e->func, BLOCK, e->dyn_smem) != cudaSuccess || n < 1) {
       (void)cudaGetLastError();
       n = 1;

@@ -68,6 +68,8 @@ static int noalloc_table(const KernelEntry* e, int64_t m, int sms, LayerTable* l
   }
   lt->tiles_total = (int)tiles;
   int per_sm = 0;
+  // static + dynamic shared memory can exceed the 48 KB default: raise the limit before asking for the occupancy
+  if (e->dyn_smem > 0) (void)cudaFuncSetAttribute(e->func, cudaFuncAttributeMaxDynamicSharedMemorySize, e->dyn_smem);
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, e->func, BLOCK, e->dyn_smem) != cudaSuccess || per_sm < 1) {
     (void)cudaGetLastError();
     per_sm = 1;
