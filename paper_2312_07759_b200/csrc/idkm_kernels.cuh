@@ -93,7 +93,8 @@ struct PassCfg {
   static constexpr int PLEN = KP * (NACC > 0 ? NACC : 1);
   static constexpr int GROUPS = BLOCK / LPW;
   static constexpr int VEC = (LPW == 1) ? 4 / D : 1;              // weight-vectors per 128-bit load
-  static constexpr int UNROLL = (LPW == 1) ? ((KPL * D >= 32) ? 1 : 2) : 1;
+  // 128-bit loads in flight per thread (thread-per-weight layouts): small codebooks are bound by memory latency
+  static constexpr int UNROLL = (LPW == 1) ? ((KPL * D >= 32) ? 1 : ((KPL * D >= 16) ? 2 : 4)) : 1;
   // weight-vectors per group per tile (bounded so that the staging buffers stay a few KB)
   static constexpr int WPG = (LPW == 1) ? VEC * UNROLL : (LPW >= 16 ? 16 : (LPW == 8 ? 8 : 4));
   static constexpr int TILE = GROUPS * WPG;
@@ -104,7 +105,10 @@ struct PassCfg {
   static constexpr int SPILL_TILES = (64 / WPG) > 0 ? (64 / WPG) : 1;
   static constexpr int DYN_SMEM = (NACC > 0) ? BLOCK * KPL * NACC * 4 : 0;
   // resident blocks per SM the register budget is sized for (the 32-lane layouts hold 8 centroids per lane)
-  static constexpr int MIN_BLOCKS = (LPW == 32) ? 2 : 1;
+  // (thread-per-weight: estimated from the registers that hold centroids, per-centroid constants and sums)
+  static constexpr int REGS_EST = KPL * ((MODE == STEP || MODE == FINAL) ? 2 * D + 1 : 3 * D + 1) + 40;
+  static constexpr int MIN_BLOCKS =
+      (LPW == 32) ? 2 : ((LPW > 1) ? 1 : ((256 / REGS_EST) > 4 ? 4 : ((256 / REGS_EST) < 1 ? 1 : (256 / REGS_EST))));
 };
 
 // ---- special-function-unit wrappers ------------------------------------------------------------
