@@ -956,10 +956,12 @@ __global__ void __launch_bounds__(BLOCK) idkm_step_precise(const __grid_constant
     if (!layer_active) continue;
     const long long row0 = p.lt.row_off[layer];
     const long long rows = p.lt.row_off[layer + 1] - row0;
-    const long long gbase = (long long)(tile - p.lt.tile_off[layer]) * TILE + (long long)grp * WPG;
-#pragma unroll 1
+    // thread-per-weight (LPW == 1): consecutive threads take consecutive rows (coalesced); otherwise a group walks
+    // its own WPG consecutive rows
+    const long long tb = (long long)(tile - p.lt.tile_off[layer]) * TILE;
+#pragma unroll 2
     for (int q = 0; q < WPG; ++q) {
-      const long long loc = gbase + q;
+      const long long loc = (LPW == 1) ? tb + (long long)q * BLOCK + grp : tb + (long long)grp * WPG + q;
       const bool ok = (loc < rows);
       const long long grow = row0 + (ok ? loc : 0);
       double w[D];
