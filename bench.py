@@ -111,6 +111,22 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+def max_over_ranks(x: float, device=None) -> float:
+    """Maximum of a per-rank number over the process group (the rank's own value without one)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(rows_per_rank: int, iterations: int, world: int, ms_per_step: float) -> float:
+    """Whole-job weight-iterations/sec: every rank runs its own replica (no exchange step on the path), the step
+    time is the slowest rank's."""
+    return world * rows_per_rank * iterations / (ms_per_step * 1e-3)
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -247,12 +263,9 @@ def main():
     n_launch = ctx.launches - launches_before[0]
     step_ms = [a.elapsed_time(b) for a, b in ev]
     total_ms = float(sum(step_ms))
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * m * (T_f + T_a) / (ms_per_step * 1e-3)
+    value = job_value(m, T_f + T_a, world, ms_per_step)
 
     info = ctx.info()
     ph = {key: float(np.mean([p[key] for p in phases])) for key in phases[0]}
@@ -304,11 +317,8 @@ def main():
                                layer_offsets=offs, out=outs)
         torch.cuda.synchronize()
         e2e_s = (time.perf_counter() - t0) / n_e2e
-        te = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        e2e_s = float(te.item())
-        e2e = {"value": world * m * (T_f + T_a) / e2e_s, "unit": "weight-iterations/s",
+        e2e_s = max_over_ranks(e2e_s, dev)
+        e2e = {"value": job_value(m, T_f + T_a, world, e2e_s * 1e3), "unit": "weight-iterations/s",
                "h2d_bytes_per_step": int(hW.numel() * 4 + hG.numel() * 4 + hC0.numel() * 4),
                "d2h_bytes_per_step": int(2 * hW.numel() * 4 + 2 * hC0.numel() * 4), "ms_per_step": e2e_s * 1e3,
                "api": "idkm_quantize_host (forward + implicit backward, pinned host buffers)"}
