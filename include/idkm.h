@@ -87,7 +87,10 @@ size_t idkm_workspace_bytes(int64_t m_total, int d, int k, int n_layers);
  * below tol, or max_iter applications were made (tol = 0: exactly max_iter applications;
  * max_iter = 0: C_out = C0).  The loop runs on the device: each application is one fused launch
  * that never stores the m x k attention matrix, and the convergence test is made by the device
- * without a host round trip (launches queued after convergence return at once).  A cluster whose
+ * without a host round trip per iteration (launches queued after convergence return at once; with
+ * tol > 0 the host queues 16 iterations at a time, peeks at a flag the device sets when every layer
+ * has converged and stays at most 32 iterations ahead of the device, so such a call may block the
+ * calling thread until the loop is within 32 iterations of its end).  A cluster whose
  * column sum is below 1e-20 keeps its centroid.  Then one final pass at the returned centroids
  * writes Wq = A C (Wq_out, may be NULL), optionally A itself (A_out, may be NULL: m*k floats, the
  * paper's O(m 2^b) term), and stashes S_j = sum_i A_ij and F(C, W)_j in the workspace.

@@ -163,6 +163,12 @@ struct idkm_ctx {
   bool timing;
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
+  // bounded run-ahead of the tolerance-mode loops: a pinned host word the device sets when all layers are done
+  int* h_flag;
+  int* d_flag;
+  int call_id;
+  cudaEvent_t chunk_ev[2];
+  bool chunk_ev_ok;
   cudaEvent_t ev[8];   // fwd: 0 start, 1 after init, 2 after steps, 3 after final; bwd: 4 start, 5 grad, 6 adj, 7 scatter
 };
 
@@ -232,6 +238,39 @@ static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p)
   p->k = ctx->k;
 }
 
+// Loops with a tolerance are queued in chunks of RUN_CHUNK iterations.  After each chunk the host peeks at the pinned
+// word the device sets once every layer's loop has ended, and it waits for the chunk before the previous one, so it
+// is never more than two chunks ahead of the device: a loop that converges early leaves at most 2 * RUN_CHUNK launches
+// that return at once instead of (cap - iterations).  The convergence decision itself stays on the device; with
+// tol = 0 everything is queued without any wait.
+constexpr int RUN_CHUNK = 16;
+
+struct RunAhead {
+  idkm_ctx* ctx;
+  bool on;
+  int chunks;
+  void begin(idkm_ctx* c, PassParams* p, bool tol_mode) {
+    ctx = c;
+    on = tol_mode && c->h_flag != nullptr && c->chunk_ev_ok;
+    chunks = 0;
+    p->host_flag = on ? c->d_flag : nullptr;
+    p->call_id = on ? ++c->call_id : 0;
+    if (on && c->call_id == 0x7fffffff) c->call_id = 0;
+  }
+  // call after iteration `it` (0-based) has been queued; true = stop queueing
+  bool after(int it) {
+    if (!on || (it + 1) % RUN_CHUNK != 0) return false;
+    cudaEventRecord(ctx->chunk_ev[chunks & 1], ctx->stream);
+    ++chunks;
+    if (*reinterpret_cast<volatile int*>(ctx->h_flag) == ctx->call_id) return true;
+    if (chunks >= 2) {
+      cudaEventSynchronize(ctx->chunk_ev[chunks & 1]);   // the chunk before the one just queued
+      if (*reinterpret_cast<volatile int*>(ctx->h_flag) == ctx->call_id) return true;
+    }
+    return false;
+  }
+};
+
 // The forward loop: every iteration launches the fp32 step and the fp64 step; each layer is taken by exactly one
 // of them (LayerState::precise), the other returns at once for it.
 static int launch_step_loop(idkm_ctx* ctx, PassParams* p, int repeat) {
@@ -243,12 +282,18 @@ static int launch_step_loop(idkm_ctx* ctx, PassParams* p, int repeat) {
   if (rc != IDKM_OK) return rc;
   rc = build_table(ctx, STEP_PRECISE, f64, &q.lt);
   if (rc != IDKM_OK) return rc;
+  RunAhead ra;
+  ra.begin(ctx, p, p->tol > 0.f);
+  q.host_flag = p->host_flag;
+  q.call_id = p->call_id;
   for (int it = 0; it < repeat; ++it) {
     p->iter = q.iter = it;
     if (e32->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
     if (e64->launch(q, q.lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
     ctx->launches += 2;
+    if (ra.after(it)) break;
   }
+  p->host_flag = nullptr;
   return IDKM_OK;
 }
 
@@ -257,10 +302,14 @@ static int launch_pass(idkm_ctx* ctx, int mode, PassParams* p, int repeat) {
   const KernelEntry* e = kernel_entry(mode, ctx->d, f);
   const int rc = build_table(ctx, mode, f, &p->lt);
   if (rc != IDKM_OK) return rc;
+  RunAhead ra;
+  ra.begin(ctx, p, mode == ADJ && p->tol > 0.f && repeat > 1);
   for (int it = 0; it < repeat; ++it) {
     if (e->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
     ++ctx->launches;
+    if (ra.after(it)) break;
   }
+  p->host_flag = nullptr;
   return IDKM_OK;
 }
 
@@ -277,6 +326,22 @@ int idkm_create(idkm_ctx** out) {
     delete c;
     return IDKM_ERR_CUDA;
   }
+  // optional: without mapped pinned memory the tolerance-mode loops simply queue every iteration
+  if (cudaHostAlloc(reinterpret_cast<void**>(&c->h_flag), sizeof(int), cudaHostAllocMapped) == cudaSuccess) {
+    *c->h_flag = 0;
+    if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->d_flag), c->h_flag, 0) != cudaSuccess) {
+      cudaFreeHost(c->h_flag);
+      c->h_flag = c->d_flag = nullptr;
+    }
+  } else {
+    c->h_flag = c->d_flag = nullptr;
+  }
+  (void)cudaGetLastError();
+  if (c->h_flag && cudaEventCreateWithFlags(&c->chunk_ev[0], cudaEventDisableTiming) == cudaSuccess) {
+    if (cudaEventCreateWithFlags(&c->chunk_ev[1], cudaEventDisableTiming) == cudaSuccess) c->chunk_ev_ok = true;
+    else cudaEventDestroy(c->chunk_ev[0]);
+  }
+  (void)cudaGetLastError();
   *out = c;
   return IDKM_OK;
 }
@@ -284,6 +349,11 @@ int idkm_create(idkm_ctx** out) {
 void idkm_destroy(idkm_ctx* ctx) {
   if (!ctx) return;
   if (ctx->hbuf) cudaFree(ctx->hbuf);
+  if (ctx->chunk_ev_ok) {
+    cudaEventDestroy(ctx->chunk_ev[0]);
+    cudaEventDestroy(ctx->chunk_ev[1]);
+  }
+  if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
   if (ctx->ev_ok)
     for (int i = 0; i < 8; ++i) cudaEventDestroy(ctx->ev[i]);
   delete ctx;

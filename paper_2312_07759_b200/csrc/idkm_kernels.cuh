@@ -80,6 +80,8 @@ struct PassParams {
   double inv_tau_d;   // 1 / tau in double (fp64 step)
   int k;
   int max_iter;       // iteration cap of the loop (for the advisory status)
+  int* host_flag;     // device view of a pinned host word, or null: set to call_id once every layer's loop has ended
+  int call_id;
   int iter;           // index of this forward iteration: a layer is stepped only while fwd_iters == iter, so that
                       // the fp32 and the fp64 step launched for the same iteration never both take it
   LayerTable lt;
@@ -365,6 +367,22 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
         st->adj_done = 1;
       } else if (p.tol > 0.f && it >= p.max_iter && st->status == ST_OK) {
         st->status = ST_MAXITER;
+      }
+    }
+    // Tell the host (it only peeks, it never waits on this) when the loops of ALL layers have ended, so that it can
+    // stop queueing iterations that would return at once.  Whichever epilogue sees every flag set writes the word.
+    if constexpr (MODE == STEP || MODE == ADJ) {
+      if (p.host_flag != nullptr && ((MODE == STEP) ? st->fwd_done : st->adj_done)) {
+        __threadfence();
+        bool all = true;
+        for (int q = 0; q < p.lt.n_layers; ++q) {
+          const volatile LayerState* sq = p.st + q;
+          all = all && (((MODE == STEP) ? sq->fwd_done : sq->adj_done) != 0);
+        }
+        if (all) {
+          *reinterpret_cast<volatile int*>(p.host_flag) = p.call_id;
+          __threadfence_system();
+        }
       }
     }
   }
