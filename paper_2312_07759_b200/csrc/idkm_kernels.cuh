@@ -98,7 +98,9 @@ struct PassCfg {
   // 128-bit loads in flight per thread (thread-per-weight layouts): small codebooks are bound by memory latency
   static constexpr int UNROLL = (LPW == 1) ? ((KPL * D >= 32) ? 1 : ((KPL * D >= 16) ? 2 : 4)) : 1;
   // weight-vectors per group per tile (bounded so that the staging buffers stay a few KB)
-  static constexpr int WPG = (LPW == 1) ? VEC * UNROLL : (LPW >= 16 ? 16 : (LPW == 8 ? 8 : 4));
+  // (thread-per-weight: one 128-bit load per thread per tile; a block takes up to UNROLL consecutive tiles at once,
+  // so small layers still spread over many blocks)
+  static constexpr int WPG = (LPW == 1) ? VEC : (LPW >= 16 ? 16 : (LPW == 8 ? 8 : 4));
   static constexpr int TILE = GROUPS * WPG;
   // Each thread's sums are moved out of its registers into a private fp32 slot in (dynamic) shared memory every
   // SPILL_TILES tiles, i.e. after about 64 weight-vectors.  A long-running fp32 accumulator silently drops the
@@ -688,8 +690,13 @@ idkm_pass(const __grid_constant__ PassParams p) {
   fetch(t_lo, layer);
 
   // ---- persistent loop over this block's tiles -------------------------------------------------
-  for (int tile = t_lo; tile < t_hi; ++tile) {
+  int adv = 1;   // tiles consumed per trip: 1, or up to UNROLL consecutive tiles of one layer (thread-per-weight)
+  for (int tile = t_lo; tile < t_hi; tile += adv) {
     while (p.lt.tile_off[layer + 1] <= tile) ++layer;
+    if constexpr (LPW == 1) {
+      const int lim = (t_hi < p.lt.tile_off[layer + 1]) ? t_hi : p.lt.tile_off[layer + 1];
+      adv = (lim - tile < Cfg::UNROLL) ? lim - tile : Cfg::UNROLL;
+    }
     if (layer != cur_layer) {
       if (cur_layer >= 0 && layer_active) flush(cur_layer);
       cur_layer = layer;
@@ -736,7 +743,8 @@ idkm_pass(const __grid_constant__ PassParams p) {
       // issue all loads of the tile first
 #pragma unroll
       for (int un = 0; un < UN; ++un) {
-        const long long loc = tbase + (long long)(un * BLOCK + tid) * VEC;
+        // trips shorter than UNROLL tiles mark the missing tiles as out of range
+        const long long loc = (un < adv) ? tbase + (long long)(un * BLOCK + tid) * VEC : rows;
         first[un] = loc;
         const long long grow = row0 + loc;
         if (vec_ok && loc + VEC <= rows) {
@@ -844,7 +852,8 @@ idkm_pass(const __grid_constant__ PassParams p) {
       }
     }
     if constexpr (ACCUM) {
-      if (++since_spill == Cfg::SPILL_TILES) {
+      since_spill += adv;
+      if (since_spill >= Cfg::SPILL_TILES) {
         spill();
         since_spill = 0;
       }
@@ -862,7 +871,7 @@ struct PreciseCfg {
   static constexpr int KP = KPL * LPW;
   static constexpr int NA = D + 1;
   static constexpr int PLEN = KP * NA;
-  static constexpr int WPG = 16;
+  static constexpr int WPG = (LPW == 1) ? 4 : 16;   // small tiles in the thread-per-weight layouts spread small layers
   static constexpr int TILE = (BLOCK / LPW) * WPG;
 };
 
