@@ -257,3 +257,38 @@ def test_config4_full_size_against_stored_oracle_state():
     # invariants that hold at any size: rows of Wq lie in the bounding box of C; sum_j S_j = m
     assert np.all(out["Wq"] >= out["C"].min(0) - 1e-6) and np.all(out["Wq"] <= out["C"].max(0) + 1e-6)
     np.testing.assert_allclose(st["S"].sum(), wl.m, rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# scaling-sweep points (fifth configuration): parity at a fixed, small iteration count
+# ----------------------------------------------------------------------------------------------------------------
+SWEEP_POINTS = [
+    (1 << 20, 1, 1, 0.01), (1 << 20, 1, 2, 0.001), (1 << 20, 1, 4, 0.01), (1 << 20, 1, 8, 0.01),
+    (1 << 20, 2, 2, 0.01), (1 << 20, 2, 4, 0.001), (1 << 20, 2, 8, 0.01),
+    (1 << 20, 4, 1, 0.001), (1 << 20, 4, 4, 0.001), (1 << 20, 4, 8, 0.001),
+    (1 << 20, 1, 2, 0.1), (1 << 20, 4, 4, 0.1),            # collapsing: the fp64 step takes over
+    (1 << 24, 1, 2, 0.01), (1 << 24, 2, 4, 0.01),
+]
+
+
+@pytest.mark.parametrize("m,d,b,tau", SWEEP_POINTS)
+def test_sweep_point_fixed_iterations(m, d, b, tau):
+    wl = WL.config5_point(m, d, b, tau)
+    wl.tol, wl.adj_tol = 0.0, 0.0
+    wl.max_iter, wl.adj_max_iter = (12, 5) if tau >= 0.1 else (5, 5)
+    ref = oracle_run(wl, mode="implicit")
+    out = gpu_run(wl, mode="implicit")
+    assert out["info"][0].status == 0
+    assert_close(out["C"], ref["C"], TOL_C, "C")
+    assert_close(out["Wq"], ref["Wq"], TOL_C, "Wq")
+    nx = kink_crossings(wl.W, out["C"], ref["C"])
+    assert_grad_close(out["dC"], ref["dC"], "dC", nx, TOL_GRAD, TOL_GRAD_KINK)
+    assert_grad_close(out["dW"], ref["dW"], "dW", nx, TOL_GRAD, TOL_GRAD_KINK)
+    # invariants that hold at any size
+    assert np.all(out["Wq"] >= out["C"].min(0) - 1e-6) and np.all(out["Wq"] <= out["C"].max(0) + 1e-6)
+    if nx:
+        wc = at_centroids(wl, ref["C"])
+        refc = oracle_backward_at(wc, wc.C0, mode="implicit")
+        outc = gpu_run(wc, mode="implicit", ctx=out["ctx"])
+        assert_close(outc["dC"], refc["dC"], TOL_GRAD, "dC at common C")
+        assert_close(outc["dW"], refc["dW"], TOL_GRAD, "dW at common C")
