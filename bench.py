@@ -189,7 +189,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4")
-    ap.add_argument("--cpu-rows", type=int, default=1 << 19)
+    ap.add_argument("--cpu-rows", type=int, default=1 << 19, help="rows of the workload the oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--iters", type=int, default=0, help="override the forward and adjoint iteration counts "
@@ -325,9 +325,9 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, sec, thr, vf, va = time_oracle_sample(wl, args.cpu_rows, 4, 4)
+        v, sec, thr, vf, va = time_oracle_sample(wl, 2 * args.cpu_rows, 10, 10)     # about 10-20 s of CPU work
         cpu = {"value": v, "unit": "weight-iterations/s", "cores": thr, "kind": "oracle",
-               "sample": f"first {min(args.cpu_rows, m)} rows of {wl.name}, 4 forward + 4 adjoint iterations, {sec:.1f} s",
+               "sample": f"first {min(2 * args.cpu_rows, m)} rows of {wl.name}, 10 forward + 10 adjoint iterations, {sec:.1f} s",
                "forward_value": vf, "adjoint_value": va}
 
     if rank == 0:
