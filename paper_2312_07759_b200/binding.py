@@ -60,6 +60,8 @@ lib.idkm_get_phase_ms.argtypes = [_vp, C.POINTER(C.c_float)]
 lib.idkm_get_phase_ms.restype = C.c_int
 lib.idkm_step_noalloc.argtypes = [_fp, C.c_int64, C.c_int, _fp, C.c_int, C.c_float, _fp, _vp]
 lib.idkm_step_noalloc.restype = C.c_int
+lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
+lib.idkm_set_adjoint_method.restype = C.c_int
 lib.idkm_launch_count.argtypes = [_vp]
 lib.idkm_launch_count.restype = C.c_int64
 lib.idkm_status_string.argtypes = [C.c_int]
@@ -222,6 +224,10 @@ class Context:
         _check(rc)
         self.n_layers = L
         return Cout, Wq, dW, dC, list(infos)
+
+    def set_adjoint_method(self, method: int) -> None:
+        """0: explicit Jacobian for k*d <= 8 (default); 1: always one fused pass per adjoint step."""
+        _check(lib.idkm_set_adjoint_method(self._h, int(method)))
 
     def set_timing(self, enable: bool = True) -> None:
         _check(lib.idkm_set_timing(self._h, 1 if enable else 0))

@@ -20,6 +20,7 @@ extern const KernelEntry k_table_grad[3][N_FAMILY];
 extern const KernelEntry k_table_adj[3][N_FAMILY];
 extern const KernelEntry k_table_scatter[3][N_FAMILY];
 extern const KernelEntry k_table_step_precise[3][N_FAMILY];
+extern const KernelEntry k_table_jacobian[3][N_FAMILY];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
@@ -61,6 +62,7 @@ const KernelEntry* kernel_entry(int mode, int d, int family) {
     case ADJ: return &k_table_adj[di][family];
     case SCATTER: return &k_table_scatter[di][family];
     case STEP_PRECISE: return &k_table_step_precise[di][family];
+    case JACOBIAN: return &k_table_jacobian[di][family];
   }
   return nullptr;
 }
@@ -88,14 +90,14 @@ int pick_family(int mode, int d, int k) {
   const int forced = forced_family(mode);
   if (forced >= 0) {
     const KernelEntry* e = kernel_entry(mode, d, forced);
-    if (e && e->kpl * e->lpw >= k) return forced;
+    if (e && e->launch && e->kpl * e->lpw >= k) return forced;
   }
   // forward step with more than 128 centroids: the 8-centroids-per-lane, full-warp layout at two blocks per SM
   // measured 3 % faster than 16 centroids per lane on half-warps
   if (mode == STEP && k > 128) return N_FAMILY - 1;
   for (int f = 0; f < N_FAMILY; ++f) {
     const KernelEntry* e = kernel_entry(mode, d, f);
-    if (e && e->kpl * e->lpw >= k) return f;
+    if (e && e->launch && e->kpl * e->lpw >= k) return f;
   }
   return -1;
 }
@@ -122,6 +124,7 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   int plen_max = 1;
   for (int mode = STEP; mode < N_MODES; ++mode) {
     const int f = pick_family(mode, d, k);
+    if (f < 0 && mode == JACOBIAN) continue;   // only small codebooks have the explicit-Jacobian pass
     if (f < 0) return false;
     const int pl = kernel_entry(mode, d, f)->plen;
     if (pl > plen_max) plen_max = pl;
@@ -166,6 +169,7 @@ struct idkm_ctx {
   bool timing;
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
+  int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
   // bounded run-ahead of the tolerance-mode loops: a pinned host word the device sets when all layers are done
   int* h_flag;
   int* d_flag;
@@ -462,8 +466,11 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   int rc = launch_pass(ctx, GRAD, &p, 1);
   if (rc != IDKM_OK) return rc;
   mark(ctx, 5);
-  if (mode == IDKM_IMPLICIT) {
-    rc = launch_pass(ctx, ADJ, &p, adj_max_iter);
+  if (mode == IDKM_IMPLICIT && adj_max_iter > 0) {
+    if (ctx->adjoint_method == 0 && pick_family(JACOBIAN, ctx->d, ctx->k) >= 0)
+      rc = launch_pass(ctx, JACOBIAN, &p, 1);      // one pass forms J_C; the whole iteration runs on it in the epilogue
+    else
+      rc = launch_pass(ctx, ADJ, &p, adj_max_iter);
     if (rc != IDKM_OK) return rc;
   }
   mark(ctx, 6);
@@ -587,6 +594,13 @@ int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out) {
     for (int i = 0; i < 3; ++i)
       if (cudaEventElapsedTime(&ms_out[3 + i], ctx->ev[4 + i], ctx->ev[5 + i]) != cudaSuccess) return IDKM_ERR_CUDA;
   }
+  return IDKM_OK;
+}
+
+int idkm_set_adjoint_method(idkm_ctx* ctx, int method) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (method != 0 && method != 1) return IDKM_ERR_PARAM;
+  ctx->adjoint_method = method;
   return IDKM_OK;
 }
 

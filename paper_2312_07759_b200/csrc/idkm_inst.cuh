@@ -43,6 +43,18 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
         IDKM_PRECISE_ENTRY(D, 8, 16), IDKM_PRECISE_ENTRY(D, 8, 32), IDKM_PRECISE_ENTRY(D, 8, 32)  \
   }
 
+template <int D, int KPL>
+static cudaError_t launch_jacobian(const PassParams& p, int grid, cudaStream_t stream) {
+  idkm_jacobian<D, KPL><<<grid, BLOCK, 0, stream>>>(p);
+  return cudaGetLastError();
+}
+#define IDKM_JAC_ENTRY(D, KPL)                                                                    \
+  {                                                                                               \
+    &launch_jacobian<D, KPL>, (const void*)&idkm_jacobian<D, KPL>, KPL, 1, JacCfg<D, KPL>::TILE,  \
+        JacCfg<D, KPL>::PLEN, 0                                                                   \
+  }
+#define IDKM_NO_ENTRY {nullptr, nullptr, 0, 0, 1, 1, 0}
+
 // forward passes keep 16 centroids per lane, backward passes 8 (they also hold F_j and u_j/S_j)
 #define IDKM_FWD_ROW(MODE, D)                                                                     \
   {                                                                                               \

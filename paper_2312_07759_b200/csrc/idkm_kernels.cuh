@@ -29,8 +29,8 @@ constexpr int MAX_BLOCKS_PER_SM = 8;
 // fp32 resolution (w - c_j rounds away the differences between the c_j).  Such layers step in fp64.
 constexpr double PRECISE_SPAN = 0.0625;
 
-enum Mode { STEP = 0, FINAL = 1, GRAD = 2, ADJ = 3, SCATTER = 4, STEP_PRECISE = 5 };
-constexpr int N_MODES = 6;
+enum Mode { STEP = 0, FINAL = 1, GRAD = 2, ADJ = 3, SCATTER = 4, STEP_PRECISE = 5, JACOBIAN = 6 };
+constexpr int N_MODES = 7;
 
 // status values mirrored from idkm.h (device side needs only these)
 constexpr int ST_OK = 0, ST_MAXITER = 1, ST_NONFINITE = -9, ST_DIVERGED = -10;
@@ -1027,6 +1027,266 @@ __global__ void __launch_bounds__(BLOCK) idkm_step_precise(const __grid_constant
     }
   }
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
+}
+
+
+// ---- explicit Jacobian for small codebooks -------------------------------------------------------------------
+// When k d <= 8 the matrix J_C = dF/dC (k d x k d, at most 64 entries) fits in a thread's registers.  One pass over
+// W accumulates it -- J[(j,a),(l,b)] = sum_i P_ija (delta_jl - A_il) n_ilb with P_ija = A_ij (w_ia - F_ja) / (S_j tau)
+// -- and the last block then runs the WHOLE adjoint iteration u <- alpha (J^T u + g) + (1 - alpha) u on that small
+// matrix in fp64: the same iterates as one fused pass over W per step, for the cost of one pass.  This is the paper's
+// own formulation (it iterates a k x k matrix, Section 4.2) restricted to where the matrix is cheap to form.
+template <int D, int KPL>
+struct JacCfg {
+  static constexpr int KD = KPL * D;
+  static constexpr int PLEN = KD * KD;
+  static constexpr int VEC = 4 / D;
+  static constexpr int TILE = BLOCK * VEC;
+};
+
+template <int D, int KPL>
+__global__ void __launch_bounds__(BLOCK) idkm_jacobian(const __grid_constant__ PassParams p) {
+  using Cfg = JacCfg<D, KPL>;
+  constexpr int KD = Cfg::KD;
+  constexpr int PLEN = Cfg::PLEN;
+  constexpr int VEC = Cfg::VEC;
+  constexpr int TILE = Cfg::TILE;
+  constexpr int SMEM_DBL = (NWARP * PLEN > PLEN + BLOCK) ? NWARP * PLEN : PLEN + BLOCK;
+  __shared__ double sm[SMEM_DBL];
+  __shared__ int s_flag;
+
+  const int tid = threadIdx.x;
+  const int lane = tid & 31;
+  const int warp = tid >> 5;
+  const int k = p.k;
+  const int nb = p.lt.n_blocks;
+  const int b = blockIdx.x;
+  const int t_lo = tile_begin(b, p.lt.tiles_total, nb);
+  const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
+  if (t_lo >= t_hi) return;
+
+  float c[KPL][D], fj[KPL][D], ist[KPL];   // centroids, F(C_T, W)_j, 1 / (S_j tau) (0 for a dead or padding cluster)
+  float jac[KD][KD];
+  float jac_hi[KD][KD];                     // second level: the running sums are moved here every 64 rows
+  int layer = 0;
+  while (p.lt.tile_off[layer + 1] <= t_lo) ++layer;
+  int cur_layer = -1;
+  bool layer_active = false;
+  int since = 0;
+
+  auto finish = [&](int l) {
+#pragma unroll
+    for (int r = 0; r < KD; ++r)
+#pragma unroll
+      for (int q = 0; q < KD; ++q) {
+        double v = (double)jac_hi[r][q] + (double)jac[r][q];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) sm[warp * PLEN + r * KD + q] = v;
+      }
+    __syncthreads();
+    double* mine = p.partials + (size_t)(b + l) * PLEN;
+    for (int o = tid; o < PLEN; o += BLOCK) {
+      double s = 0.0;
+#pragma unroll
+      for (int wv = 0; wv < NWARP; ++wv) s += sm[wv * PLEN + o];
+      mine[o] = s;
+    }
+    __threadfence();
+    __syncthreads();
+    const int first_b = block_of_tile(p.lt.tile_off[l], p.lt.tiles_total, nb);
+    const int last_b = block_of_tile(p.lt.tile_off[l + 1] - 1, p.lt.tiles_total, nb);
+    const int n_contrib = last_b - first_b + 1;
+    if (tid == 0) {
+      const unsigned int prev = atomicAdd(&p.st[l].ticket, 1u);
+      s_flag = (prev == (unsigned int)(n_contrib - 1));
+    }
+    __syncthreads();
+    if (!s_flag) return;
+    __threadfence();
+    // second level in slot order: PLEN <= 64 outputs, BLOCK / PLEN strided chunks each, then the chunks in order
+    double* tot = sm;            // [PLEN]
+    double* scratch = sm + PLEN; // [BLOCK]
+    const double* base = p.partials + (size_t)(first_b + l) * PLEN;
+    constexpr int NCH = BLOCK / PLEN;
+    {
+      const int ch = tid / PLEN, o = tid % PLEN;
+      double s = 0.0;
+      if (ch < NCH)
+        for (int q = ch; q < n_contrib; q += NCH) s += __ldcg(base + (size_t)q * PLEN + o);
+      __syncthreads();
+      scratch[tid] = s;
+      __syncthreads();
+      if (tid < PLEN) {
+        double r2 = 0.0;
+        for (int c2 = 0; c2 < NCH; ++c2) r2 += scratch[c2 * PLEN + tid];
+        tot[tid] = r2;
+      }
+      __syncthreads();
+    }
+    if (warp == 0) {
+      // The iteration on the small matrix, by one warp: lane q < n owns coordinate q of u and column q of J
+      // (J^T u)_q = sum_r J[r][q] u_r; u_r is fetched from lane r by a shuffle.  All lanes see the same residual.
+      LayerState* st = p.st + l;
+      const int n = k * D;
+      const int q = lane;
+      double jcol[KD];
+#pragma unroll
+      for (int r = 0; r < KD; ++r) jcol[r] = (q < n && r < n) ? tot[r * KD + q] : 0.0;
+      const double g = (q < n) ? (double)p.gvec[(size_t)l * n + q] : 0.0;
+      double u = g;
+      const double al = (double)p.alpha;
+      int it = 0, up = 0, status = st->status, done = 0;
+      float res = 0.f, prev = 3.0e38f;
+      while (it < p.max_iter && !done) {
+        double s = 0.0;
+#pragma unroll
+        for (int r = 0; r < KD; ++r) s = fma(jcol[r], __shfl_sync(0xffffffffu, u, r), s);
+        const double un = (q < n) ? al * (s + g) + (1.0 - al) * u : 0.0;
+        double num = (un - u) * (un - u), den = un * un;
+        double badv = (!(un == un) || fabs(un) > 1e300) ? 1.0 : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          num += __shfl_xor_sync(0xffffffffu, num, o);
+          den += __shfl_xor_sync(0xffffffffu, den, o);
+          badv += __shfl_xor_sync(0xffffffffu, badv, o);
+        }
+        u = un;
+        double dn = sqrt(den);
+        if (dn < 1e-300) dn = 1e-300;
+        res = (float)(sqrt(num) / dn);
+        ++it;
+        up = (res > prev) ? up + 1 : 0;
+        prev = res;
+        if (badv > 0.0 || up >= 10) {
+          status = ST_DIVERGED;
+          done = 1;
+        } else if (p.tol > 0.f && res < p.tol) {
+          done = 1;
+        } else if (p.tol > 0.f && it >= p.max_iter && status == ST_OK) {
+          status = ST_MAXITER;
+        }
+      }
+      if (q < n) p.u[(size_t)l * n + q] = (float)u;
+      if (lane == 0) {
+        st->ticket = 0u;
+        st->adj_iters = it;
+        st->adj_res = res;
+        st->adj_up = up;
+        st->adj_prev = prev;
+        st->adj_done = 1;
+        st->status = status;
+      }
+    }
+    __syncthreads();
+  };
+
+  for (int tile = t_lo; tile < t_hi; ++tile) {
+    while (p.lt.tile_off[layer + 1] <= tile) ++layer;
+    if (layer != cur_layer) {
+      if (cur_layer >= 0 && layer_active) finish(cur_layer);
+      cur_layer = layer;
+      layer_active = (p.st[layer].adj_done == 0);
+      since = 0;
+      if (layer_active) {
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          const float s = (t < k) ? p.S[(size_t)layer * k + t] : 0.f;
+          ist[t] = (t < k && s >= S_MIN_F) ? p.inv_tau / s : 0.f;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            c[t][a] = (t < k) ? p.C[((size_t)layer * k + t) * D + a] : PAD_COORD;
+            fj[t][a] = (t < k) ? p.F[((size_t)layer * k + t) * D + a] : 0.f;
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < KD; ++r)
+#pragma unroll
+          for (int q = 0; q < KD; ++q) {
+            jac[r][q] = 0.f;
+            jac_hi[r][q] = 0.f;
+          }
+      }
+    }
+    if (!layer_active) continue;
+    const long long row0 = p.lt.row_off[layer];
+    const long long rows = p.lt.row_off[layer + 1] - row0;
+    const long long loc0 = (long long)(tile - p.lt.tile_off[layer]) * TILE + (long long)tid * VEC;
+    const bool vec_ok = ((row0 * D) % 4 == 0) && (loc0 + VEC <= rows);
+    float wv[VEC][D];
+    if (vec_ok) {
+      const float4 x = __ldg(reinterpret_cast<const float4*>(p.W + (row0 + loc0) * D));
+      const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int v = 0; v < VEC; ++v)
+#pragma unroll
+        for (int a = 0; a < D; ++a) wv[v][a] = xs[v * D + a];
+    } else {
+#pragma unroll
+      for (int v = 0; v < VEC; ++v)
+#pragma unroll
+        for (int a = 0; a < D; ++a) wv[v][a] = (loc0 + v < rows) ? __ldg(p.W + (row0 + loc0 + v) * D + a) : 0.f;
+    }
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) {
+      const bool valid = (loc0 + v < rows);
+      float dist[KPL], rs[KPL], e[KPL];
+      (void)rs;
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        if constexpr (D == 1) {
+          dist[t] = fabsf(wv[v][0] - c[t][0]);
+        } else {
+          float sq = 1e-30f;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const float df = wv[v][a] - c[t][a];
+            sq = fmaf(df, df, sq);
+          }
+          rs[t] = rsqrt_approx(sq);
+          dist[t] = sq * rs[t];
+        }
+      }
+      const float mref = tree_reduce<KPL, 1>(dist) * p.scale;
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) e[t] = ex2_approx(fmaf(-p.scale, dist[t], mref));
+      const float r = valid ? rcp_approx(tree_reduce<KPL, 0>(e)) : 0.f;
+      float P[KD], Y[KD], Q[KD];
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        const float at = e[t] * r;
+#pragma unroll
+        for (int a = 0; a < D; ++a) {
+          const float df = wv[v][a] - c[t][a];
+          float n;
+          if constexpr (D == 1) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
+          else n = df * rs[t];
+          Q[t * D + a] = n;
+          Y[t * D + a] = at * n;
+          P[t * D + a] = at * ist[t] * (wv[v][a] - fj[t][a]);
+        }
+      }
+#pragma unroll
+      for (int rr = 0; rr < KD; ++rr)
+#pragma unroll
+        for (int q = 0; q < KD; ++q) {
+          jac[rr][q] = fmaf(-P[rr], Y[q], jac[rr][q]);
+          if (rr / D == q / D) jac[rr][q] = fmaf(P[rr], Q[q], jac[rr][q]);   // the delta_jl block
+        }
+    }
+    since += VEC;
+    if (since >= 64) {
+#pragma unroll
+      for (int rr = 0; rr < KD; ++rr)
+#pragma unroll
+        for (int q = 0; q < KD; ++q) {
+          jac_hi[rr][q] += jac[rr][q];
+          jac[rr][q] = 0.f;
+        }
+      since = 0;
+    }
+  }
+  if (cur_layer >= 0 && layer_active) finish(cur_layer);
 }
 
 // host-side dispatch (defined in the per-mode instantiation units)

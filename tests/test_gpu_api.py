@@ -88,3 +88,34 @@ def test_non_default_stream():
     s.synchronize()
     assert_close(fr.C.cpu().numpy(), ref["C"], TOL_C, "C")
     assert_close(dW.cpu().numpy(), ref["dW"], TOL_GRAD, "dW")
+
+
+@pytest.mark.parametrize("m,d,k", [(30001, 1, 4), (20000, 1, 8), (10000, 2, 4), (9000, 4, 2), (5000, 2, 3)])
+def test_explicit_jacobian_adjoint_equals_fused_passes(m, d, k):
+    """For k*d <= 8 the adjoint iteration runs on the explicitly formed k d x k d matrix (one pass over W); it must
+    give the iterates of the one-pass-per-step path, with the tolerance rule and the counters behaving the same."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(m, d, k, 0.012, std=0.03, seed=m + k, max_iter=15, adj_max_iter=12, init="rows", g_std=0.3)
+    W, C0, G = (torch.from_numpy(x).cuda() for x in (wl.W, wl.C0, wl.G))
+    res = {}
+    for method in (0, 1):
+        ctx = B.Context()
+        ctx.set_adjoint_method(method)
+        ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter)
+        before = ctx.launches
+        dW, dC = ctx.backward(G, B.IMPLICIT, 0.0, wl.adj_max_iter, 1.0)
+        info = ctx.info()[0]
+        assert info.status == 0 and info.adj_iters == wl.adj_max_iter
+        res[method] = (dW.cpu().numpy(), dC.cpu().numpy(), info.adj_residual, ctx.launches - before)
+        # tolerance mode: both stop at the same iteration (or one apart, by fp32 rounding of the residual)
+        dW2, dC2 = ctx.backward(G, B.IMPLICIT, 1e-4, 500, 0.5)
+        res[(method, "tol")] = (ctx.info()[0].adj_iters, dC2.cpu().numpy())
+    assert res[0][3] == 3 and res[1][3] == 2 + wl.adj_max_iter          # g, J (or 12 passes), dW
+    assert_close(res[0][1], res[1][1], 1e-5, "dC")
+    assert_close(res[0][0], res[1][0], 1e-5, "dW")
+    assert abs(res[0][2] - res[1][2]) <= 1e-3 * max(res[1][2], 1e-30) + 1e-9
+    assert abs(res[(0, "tol")][0] - res[(1, "tol")][0]) <= 1
+    assert_close(res[(0, "tol")][1], res[(1, "tol")][1], 1e-3, "dC at tolerance")
+    ref = oracle_run(wl)
+    assert_close(res[0][1], ref["dC"], TOL_GRAD if d > 1 else 3e-2, "dC vs oracle")

@@ -14,7 +14,7 @@ def test_library_exports_every_declared_symbol():
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     names = set(re.findall(r"\b(idkm_[a-z_0-9]+)\s*\(", header))
     assert {"idkm_create", "idkm_destroy", "idkm_forward", "idkm_forward_batched", "idkm_backward", "idkm_get_info",
-            "idkm_workspace_bytes", "idkm_quantize_host", "idkm_status_string", "idkm_launch_count", "idkm_set_timing", "idkm_get_phase_ms"} <= names
+            "idkm_workspace_bytes", "idkm_quantize_host", "idkm_status_string", "idkm_launch_count", "idkm_set_timing", "idkm_get_phase_ms", "idkm_set_adjoint_method"} <= names
     for n in names:
         assert hasattr(lib, n), n
 
