@@ -875,10 +875,8 @@ struct PreciseCfg {
   static constexpr int TILE = (BLOCK / LPW) * WPG;
 };
 
-__device__ __forceinline__ double exp_small(double y) {   // |y| <= PRECISE_SPAN: truncation error < 1e-16
-  double s = 1.0 / 40320.0;
-  s = fma(s, y, 1.0 / 5040.0);
-  s = fma(s, y, 1.0 / 720.0);
+__device__ __forceinline__ double exp_small(double y) {   // |y| <= PRECISE_SPAN: truncation error y^7/5040 < 8e-13
+  double s = 1.0 / 720.0;
   s = fma(s, y, 1.0 / 120.0);
   s = fma(s, y, 1.0 / 24.0);
   s = fma(s, y, 1.0 / 6.0);
@@ -986,43 +984,63 @@ __global__ void __launch_bounds__(BLOCK) idkm_step_precise(const __grid_constant
     // thread-per-weight (LPW == 1): consecutive threads take consecutive rows (coalesced); otherwise a group walks
     // its own WPG consecutive rows
     const long long tb = (long long)(tile - p.lt.tile_off[layer]) * TILE;
-#pragma unroll 2
-    for (int q = 0; q < WPG; ++q) {
-      const long long loc = (LPW == 1) ? tb + (long long)q * BLOCK + grp : tb + (long long)grp * WPG + q;
-      const bool ok = (loc < rows);
-      const long long grow = row0 + (ok ? loc : 0);
-      double w[D];
+    // all rows of the trip are fetched first (thread-per-weight layouts: 4 loads in flight per thread)
+    constexpr int QB = (LPW == 1) ? WPG : 2;   // rows per fully unrolled batch
+#pragma unroll 1
+    for (int q0 = 0; q0 < WPG; q0 += QB) {
+      float wf[QB][D];
+      bool okq[QB];
 #pragma unroll
-      for (int a = 0; a < D; ++a) w[a] = (double)__ldg(p.W + grow * D + a);
-      double dist[KPL];
-      double lmin = 1e300;
+      for (int qq = 0; qq < QB; ++qq) {
+        const int q = q0 + qq;
+        const long long loc = (LPW == 1) ? tb + (long long)q * BLOCK + grp : tb + (long long)grp * WPG + q;
+        okq[qq] = (loc < rows);
+        const long long grow = row0 + (okq[qq] ? loc : 0);
 #pragma unroll
-      for (int t = 0; t < KPL; ++t) {
-        double sq = 0.0;
+        for (int a = 0; a < D; ++a) wf[qq][a] = __ldg(p.W + grow * D + a);
+      }
 #pragma unroll
-        for (int a = 0; a < D; ++a) {
-          const double df = w[a] - c[t][a];
-          sq = (D == 1) ? fabs(df) : fma(df, df, sq);
+      for (int qq = 0; qq < QB; ++qq) {
+        double w[D];
+#pragma unroll
+        for (int a = 0; a < D; ++a) w[a] = (double)wf[qq][a];
+        double dist[KPL];
+        double lmin = 1e300;
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          double sq = 0.0;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const double df = w[a] - c[t][a];
+            sq = (D == 1) ? fabs(df) : fma(df, df, sq);
+          }
+          dist[t] = (D == 1) ? sq : sqrt(sq);
+          if (gl * KPL + t < k) lmin = fmin(lmin, dist[t]);
         }
-        dist[t] = (D == 1) ? sq : sqrt(sq);
-        if (gl * KPL + t < k) lmin = fmin(lmin, dist[t]);
-      }
-      const double gmin = group_min_d<LPW>(lmin);
-      double e[KPL];
-      double lsum = 0.0;
+        const double gmin = group_min_d<LPW>(lmin);
+        double e[KPL];
+        double lsum = 0.0;
 #pragma unroll
-      for (int t = 0; t < KPL; ++t) {
-        e[t] = (gl * KPL + t < k) ? exp_small((gmin - dist[t]) * p.inv_tau_d) : 0.0;
-        lsum += e[t];
-      }
-      const double gsum = group_sum_d<LPW>(lsum);
-      const double r = ok ? 1.0 / gsum : 0.0;
+        for (int t = 0; t < KPL; ++t) {
+          e[t] = (gl * KPL + t < k) ? exp_small((gmin - dist[t]) * p.inv_tau_d) : 0.0;
+          lsum += e[t];
+        }
+        const double gsum = group_sum_d<LPW>(lsum);
+        // reciprocal of the row sum (1 <= gsum <= k): fp32 seed and two Newton steps in fp64 (error ~1e-28 relative
+        // to the seed's 1e-7 squared twice), cheaper than a double division
+        double r = (double)rcp_approx((float)gsum);
+        r = r * (2.0 - gsum * r);
+        r = r * (2.0 - gsum * r);
+        if (!okq[qq]) r = 0.0;
+        double rw[D];
 #pragma unroll
-      for (int t = 0; t < KPL; ++t) {
-        const double at = e[t] * r;
-        acc[t][0] += at;
+        for (int a = 0; a < D; ++a) rw[a] = r * w[a];
 #pragma unroll
-        for (int a = 0; a < D; ++a) acc[t][1 + a] = fma(at, w[a], acc[t][1 + a]);
+        for (int t = 0; t < KPL; ++t) {
+          acc[t][0] = fma(e[t], r, acc[t][0]);
+#pragma unroll
+          for (int a = 0; a < D; ++a) acc[t][1 + a] = fma(e[t], rw[a], acc[t][1 + a]);
+        }
       }
     }
   }
