@@ -442,8 +442,17 @@ idkm_pass(const __grid_constant__ PassParams p) {
   // instructions of sm_100 were measured on this layout: they halve the issue slots of the FMAs but run on half of
   // the FMA pipe, and the step came out slower, so the arithmetic below is scalar.)
   float2 c2[KH][D];                // owned centroids
-  float us[NEED_U ? KPL : 1][D];   // u_j / S_j (0 for a dead cluster)
-  float kap[NEED_U ? KPL : 1];     // (u_j / S_j) . F(C_T, W)_j, so that p_ij = (u_j / S_j) . w_i - kap_j
+  // u_j / S_j (0 for a dead cluster) and kap_j = (u_j / S_j) . F(C_T, W)_j, so that p_ij = (u_j / S_j) . w_i - kap_j.
+  // The full-warp layouts keep them in shared memory ([t][lane] order: conflict-free), the others in registers:
+  // with 8 centroids per lane at two blocks per SM the registers do not hold them without spilling.
+  constexpr bool US_SMEM = NEED_U && (LPW == 32);
+  float us[(NEED_U && !US_SMEM) ? KPL : 1][D];
+  float kap[(NEED_U && !US_SMEM) ? KPL : 1];
+  __shared__ __align__(16) float us_sm[US_SMEM ? KPL * LPW * D : 4];
+  __shared__ float kap_sm[US_SMEM ? KPL * LPW : 1];
+  (void)us_sm; (void)kap_sm;
+  auto us_ = [&](int t, int a) -> float { return US_SMEM ? us_sm[(t * LPW + gl) * D + a] : us[US_SMEM ? 0 : t][a]; };
+  auto kap_ = [&](int t) -> float { return US_SMEM ? kap_sm[t * LPW + gl] : kap[US_SMEM ? 0 : t]; };
   float2 acc2[ACCUM ? KH : 1][NA];
   (void)kap; (void)us; (void)acc2;
   auto c_ = [&](int t, int a) -> float& { return (t & 1) ? c2[t >> 1][a].y : c2[t >> 1][a].x; };
@@ -468,10 +477,19 @@ idkm_pass(const __grid_constant__ PassParams p) {
 #pragma unroll
         for (int a = 0; a < D; ++a) {
           const float f = (j < k) ? p.F[((size_t)l * k + j) * D + a] : 0.f;
-          us[t][a] = (j < k) ? p.u[((size_t)l * k + j) * D + a] * inv : 0.f;
-          kp = fmaf(us[t][a], f, kp);
+          const float uv = (j < k) ? p.u[((size_t)l * k + j) * D + a] * inv : 0.f;
+          kp = fmaf(uv, f, kp);
+          if constexpr (US_SMEM) {
+            if (grp == 0) us_sm[(t * LPW + gl) * D + a] = uv;
+          } else {
+            us[t][a] = uv;
+          }
         }
-        kap[t] = kp;
+        if constexpr (US_SMEM) {
+          if (grp == 0) kap_sm[t * LPW + gl] = kp;
+        } else {
+          kap[t] = kp;
+        }
       }
       if constexpr (ACCUM) {
 #pragma unroll
@@ -574,9 +592,9 @@ idkm_pass(const __grid_constant__ PassParams p) {
       for (int t = 0; t < KPL; ++t) {
         float v = 0.f;
         if constexpr (NEED_U) {
-          v = -kap[t];
+          v = -kap_(t);
 #pragma unroll
-          for (int a = 0; a < D; ++a) v = fmaf(us[t][a], w[a], v);
+          for (int a = 0; a < D; ++a) v = fmaf(us_(t, a), w[a], v);
         }
         if constexpr (NEED_G) {
 #pragma unroll
@@ -603,7 +621,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
           else n = df;
           if constexpr (MODE == GRAD) acc_(t, a) = fmaf(at, gi[a], fmaf(et, n, acc_(t, a)));
           if constexpr (MODE == ADJ) acc_(t, a) = fmaf(et, n, acc_(t, a));
-          if constexpr (MODE == SCATTER) dwl[a] = fmaf(at, us[t][a], fmaf(-et, n, dwl[a]));
+          if constexpr (MODE == SCATTER) dwl[a] = fmaf(at, us_(t, a), fmaf(-et, n, dwl[a]));
         }
       }
       if constexpr (MODE == SCATTER) {
@@ -704,7 +722,9 @@ idkm_pass(const __grid_constant__ PassParams p) {
         layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise == 0) && (p.st[layer].fwd_iters == p.iter);
       else if constexpr (MODE == ADJ) layer_active = (p.st[layer].adj_done == 0);
       else layer_active = true;
+      if constexpr (US_SMEM) __syncthreads();   // the previous layer's table is no longer read
       if (layer_active) load_layer(layer);
+      if constexpr (US_SMEM) __syncthreads();   // table written by the first group, read by all
       since_spill = 0;
     }
     if constexpr (LPW > 1) {
