@@ -3,7 +3,30 @@
 #pragma once
 #include "idkm_kernels.cuh"
 
+#include <stdlib.h>
+#include <string.h>
+
 namespace idkm {
+
+// Launch with programmatic dependent launch: the next kernel of the stream may be scheduled while this one drains
+// (it waits in griddepcontrol.wait until this grid has completed and its writes are visible), which hides the launch
+// latency between the short dependent kernels of a loop.
+template <typename Kernel>
+static cudaError_t launch_pdl(Kernel kernel, const PassParams& p, int grid, int dyn_smem, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3((unsigned)grid, 1, 1);
+  cfg.blockDim = dim3(BLOCK, 1, 1);
+  cfg.dynamicSmemBytes = (size_t)dyn_smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  static const bool pdl_off = (getenv("IDKM_NO_PDL") != nullptr);   // tuning knob: plain stream order
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl_off ? 0 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, p);
+}
 
 template <int MODE, int D, int KPL, int LPW>
 static cudaError_t launch_one(const PassParams& p, int grid, cudaStream_t stream) {
@@ -15,8 +38,7 @@ static cudaError_t launch_one(const PassParams& p, int grid, cudaStream_t stream
     if (rc != cudaSuccess) return rc;
     configured = true;
   }
-  idkm_pass<MODE, D, KPL, LPW><<<grid, BLOCK, DYN, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(idkm_pass<MODE, D, KPL, LPW>, p, grid, DYN, stream);
 }
 
 #define IDKM_ENTRY(MODE, D, KPL, LPW)                                                             \
@@ -28,8 +50,7 @@ static cudaError_t launch_one(const PassParams& p, int grid, cudaStream_t stream
 
 template <int D, int KPL, int LPW>
 static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t stream) {
-  idkm_step_precise<D, KPL, LPW><<<grid, BLOCK, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(idkm_step_precise<D, KPL, LPW>, p, grid, 0, stream);
 }
 #define IDKM_PRECISE_ENTRY(D, KPL, LPW)                                                           \
   {                                                                                               \
@@ -45,8 +66,7 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
 
 template <int D, int KPL>
 static cudaError_t launch_jacobian(const PassParams& p, int grid, cudaStream_t stream) {
-  idkm_jacobian<D, KPL><<<grid, BLOCK, 0, stream>>>(p);
-  return cudaGetLastError();
+  return launch_pdl(idkm_jacobian<D, KPL>, p, grid, 0, stream);
 }
 #define IDKM_JAC_ENTRY(D, KPL)                                                                    \
   {                                                                                               \
