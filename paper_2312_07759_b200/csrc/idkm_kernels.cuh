@@ -319,19 +319,45 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
       p.u[(size_t)l * k * D + o] = (float)unew;
     }
   }
-  bad = block_sum_double(bad, scratch);
-  if constexpr (MODE == STEP || MODE == ADJ) {
-    num = block_sum_double(num, scratch);
-    den = block_sum_double(den, scratch);
-  }
+  // All block-wide reductions of the epilogue in one go (two barriers): warp trees by shuffle, then the NWARP warp
+  // results combined in warp order by every thread.  Slots: bad, num, den, dead (sums), cmin[D] (min), cmax[D] (max).
   double box2 = 0.0;
-  if constexpr (MODE == STEP) {
-    dead = block_sum_double(dead, scratch);
+  {
+    constexpr int NV = 4 + 2 * D;
+    double v[NV];
+    v[0] = bad; v[1] = num; v[2] = den; v[3] = dead;
 #pragma unroll
     for (int a = 0; a < D; ++a) {
-      const double lo = block_reduce_double<1>(cmin[a], scratch);
-      const double hi = block_reduce_double<2>(cmax[a], scratch);
-      box2 += (hi - lo) * (hi - lo);
+      v[4 + a] = cmin[a];
+      v[4 + D + a] = cmax[a];
+    }
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const double other = __shfl_xor_sync(0xffffffffu, v[i], o);
+        v[i] = (i < 4) ? v[i] + other : ((i < 4 + D) ? fmin(v[i], other) : fmax(v[i], other));
+      }
+    }
+    __syncthreads();
+    if ((tid & 31) == 0) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) scratch[(tid >> 5) * NV + i] = v[i];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      double r = scratch[i];
+      for (int wv = 1; wv < NWARP; ++wv) {
+        const double other = scratch[wv * NV + i];
+        r = (i < 4) ? r + other : ((i < 4 + D) ? fmin(r, other) : fmax(r, other));
+      }
+      v[i] = r;
+    }
+    bad = v[0]; num = v[1]; den = v[2]; dead = v[3];
+    if constexpr (MODE == STEP) {
+#pragma unroll
+      for (int a = 0; a < D; ++a) box2 += (v[4 + D + a] - v[4 + a]) * (v[4 + D + a] - v[4 + a]);
     }
   }
   if (tid == 0) {
