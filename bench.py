@@ -60,6 +60,15 @@ def pair_ops(d: int):
     return 3 * d + 5, 2      # d sub, d fma (square), mul(D), min, fma, add, fma(S), d fma(N)  + rsqrt, ex2
 
 
+def adjoint_pair_ops(d: int):
+    """Algorithmic work of one fused adjoint step per pair (Eq. 14's vector-Jacobian product): the softmax of the
+    forward step without its S / N sums, then p_ij (d fma), its attention-weighted mean (fma), e_ij(p) / (tau D_ij)
+    (sub, 3 mul; 2 mul and a sign for d = 1) and the d sums of e_ij n_ij."""
+    if d == 1:
+        return 11, 1         # sub|abs, min, fma, add, fma(p), fma(mean), sub, mul, mul, sign, fma  + ex2
+    return 4 * d + 9, 2      # d sub, d fma, mul(D), min, fma, add, d fma(p), fma(mean), sub, 3 mul, d fma  + rsqrt, ex2
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML while the timed region runs."""
 
@@ -297,6 +306,26 @@ def main():
     # caches before the launch, so this is the cold-L2 figure); only known for the profiled workload
     roof["traffic"] = 67.20e6 + 1.24e6 if wl.name.startswith("cfg4_vq_m4194304") and args.iters == 0 else None
     roof["roofline_ms"] = max(t_hbm, t_fp32, t_sfu) * 1e3
+    # the same two pipes measured now by the library's register-only micro-benchmarks (at the clock of an otherwise
+    # idle GPU): the nominal peak above is the contract figure, this one shows how much of it the hardware delivers
+    fp32_rate, sfu_rate = B.measure_pipe_rates()
+    roof["pipes_measured"] = {"fp32_lane_ops_per_s": fp32_rate, "sfu_lane_ops_per_s": sfu_rate,
+                              "fp32_lanes_per_clk_per_sm_at_max_clock": fp32_rate / (SM_COUNT * SM_MAX_MHZ * 1e6),
+                              "sfu_lanes_per_clk_per_sm_at_max_clock": sfu_rate / (SM_COUNT * SM_MAX_MHZ * 1e6)}
+    roof["frac_of_measured_pipes"] = max(t_hbm, pairs * fp32_ops / fp32_rate, pairs * sfu_ops / sfu_rate) \
+        / (step_kernel_ms * 1e-3)
+    # the adjoint step takes the larger share of the step's time: the same arithmetic for it
+    a_fp32, a_sfu = adjoint_pair_ops(d)
+    ta_fp32 = pairs * a_fp32 / (SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6)
+    ta_sfu = pairs * a_sfu / (SM_COUNT * SFU_LANES_PER_SM * SM_MAX_MHZ * 1e6)
+    ta = max(t_hbm, ta_fp32, ta_sfu)
+    roof_adj = None
+    if T_a > 0 and adj_kernel_ms > 0:
+        roof_adj = {"kernel": "idkm_pass<ADJ> (fused adjoint step)", "kernel_ms": adj_kernel_ms, "roofline_ms": ta * 1e3,
+                    "bound": "hbm" if ta == t_hbm else "alu", "frac": ta / (adj_kernel_ms * 1e-3),
+                    "fp32_ops_per_pair": a_fp32, "sfu_ops_per_pair": a_sfu,
+                    "note": "only meaningful where the fused passes run the iteration (k d > 8); the explicit-Jacobian "
+                            "path makes one pass over W for the whole solve"}
 
     # ---- end to end through the host-buffer entry point ----------------------------------------------------------
     e2e = None
@@ -342,7 +371,7 @@ def main():
             "forward_wit_per_s": world * m * T_f / (ph["steps"] * 1e-3) if T_f else None,
             "adjoint_wit_per_s": world * m * T_a / (ph["adjoint"] * 1e-3) if T_a else None,
             "phase_ms": ph, "step_kernel_ms": step_kernel_ms, "adjoint_kernel_ms": adj_kernel_ms,
-            "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(n_launch), "clocks": clocks,
+            "roofline": roof, "roofline_adjoint": roof_adj, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(n_launch), "clocks": clocks,
             "info": {"status": [i.status for i in info][:4], "fwd_residual": info[0].fwd_residual,
                      "adj_residual": info[0].adj_residual},
         }

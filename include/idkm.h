@@ -196,6 +196,17 @@ int idkm_step_noalloc(const float* W, int64_t m, int d, const float* C_in, int k
  */
 int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
 
+/*
+ * Measured issue rates of the two pipes that bound the arithmetic-bound passes, for roofline denominators (the
+ * paper has no counterpart: this is a measurement utility, nothing on the IDKM path calls it).  Two register-only
+ * kernels over all SMs -- eight independent chains per thread of fp32 fused multiply-adds, and of ex2.approx --
+ * are timed with CUDA events on cuda_stream (best of five after two warm-up launches, a few milliseconds in all).
+ * Writes, to HOST doubles, lane-operations per second: one fused multiply-add (counted as one operation, not two
+ * flops) resp. one special-function result, per lane.  The figures are at the clock the GPU ran during the
+ * measurement.  Synchronises cuda_stream.  Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_CUDA.
+ */
+int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_per_s, void* cuda_stream);
+
 /* Number of kernels this ctx has launched since idkm_create (for accounting in benchmarks). */
 int64_t idkm_launch_count(const idkm_ctx* ctx);
 

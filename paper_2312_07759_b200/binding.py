@@ -64,6 +64,8 @@ lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
 lib.idkm_set_adjoint_method.restype = C.c_int
 lib.idkm_launch_count.argtypes = [_vp]
 lib.idkm_launch_count.restype = C.c_int64
+lib.idkm_measure_pipe_rates.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), _vp]
+lib.idkm_measure_pipe_rates.restype = C.c_int
 lib.idkm_status_string.argtypes = [C.c_int]
 lib.idkm_status_string.restype = C.c_char_p
 
@@ -116,6 +118,13 @@ def step_noalloc(W, C_in, tau: float, C_out=None, stream=None):
     _check(lib.idkm_step_noalloc(_ptr(W), int(W.shape[0]), int(W.shape[1]), _ptr(C_in), int(C_in.shape[0]),
                                  float(tau), _ptr(C_out), _stream(stream)))
     return C_out
+
+
+def measure_pipe_rates(stream=None):
+    """``idkm_measure_pipe_rates``: (fp32 FMA lane-operations/s, special-function lane-operations/s) measured now."""
+    a, b = C.c_double(0.0), C.c_double(0.0)
+    _check(lib.idkm_measure_pipe_rates(C.byref(a), C.byref(b), _stream(stream)))
+    return float(a.value), float(b.value)
 
 
 class Context:

@@ -119,3 +119,18 @@ def test_explicit_jacobian_adjoint_equals_fused_passes(m, d, k):
     assert_close(res[(0, "tol")][1], res[(1, "tol")][1], 1e-3, "dC at tolerance")
     ref = oracle_run(wl)
     assert_close(res[0][1], ref["dC"], TOL_GRAD if d > 1 else 3e-2, "dC vs oracle")
+
+
+def test_pipe_rate_microbenchmarks():
+    """The measured fp32 and special-function issue rates land near the documented widths of the two pipes
+    (128 and 16 results per clock per SM): between 60 % and 105 % of width x SM count x maximum SM clock (a
+    lower clock under load or a power cap lowers the figure, nothing raises it)."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    props = torch.cuda.get_device_properties(0)
+    sms = props.multi_processor_count
+    clk_hz = 1965e6                   # maximum SM clock of the part
+    fp32, sfu = B.measure_pipe_rates()
+    assert 0.60 < fp32 / (sms * 128 * clk_hz) < 1.05, fp32
+    assert 0.60 < sfu / (sms * 16 * clk_hz) < 1.05, sfu
+    assert B.lib.idkm_measure_pipe_rates(None, None, None) == B.ERR_NULL
