@@ -176,8 +176,8 @@ int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out);
  * C_out may alias.  The result is that of idkm_forward with max_iter = 1 (same kernels, same reduction
  * order).  Asynchronous on cuda_stream.
  *
- * Limits and sharing.  Returns IDKM_ERR_NOALLOC_TOO_LARGE when (resident blocks + 1) * padded k * (d+1)
- * * 8 bytes + 256 exceeds IDKM_NOALLOC_SCRATCH_BYTES; every supported (d, k) fits on a B200, the check
+ * Limits and sharing.  Returns IDKM_ERR_NOALLOC_TOO_LARGE when (resident blocks + 1) * (1 + 1/16) * padded k
+ * * (d+1) * 8 bytes + a few KB exceeds IDKM_NOALLOC_SCRATCH_BYTES; every supported (d, k) fits on a B200, the check
  * guards larger parts.  All calls on a device share the one array, which still holds the previous call's
  * contents when the next begins: the call clears what must start at zero itself, but two calls that
  * overlap on the GPU (different streams, or different host threads) race on it -- serialise them.

@@ -24,8 +24,9 @@ extern const KernelEntry k_table_jacobian[3][N_FAMILY];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
-                                  double inv_tau) {
+                                  double inv_tau, unsigned int* gtickets, int n_groups) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  for (int o = i; o < n_groups; o += gridDim.x * blockDim.x) gtickets[o] = 0u;
   if (i < n_layers) {
     LayerState s;
     s.fwd_done = 0; s.fwd_iters = 0; s.fwd_res = 0.f; s.dead = 0;
@@ -105,8 +106,8 @@ int pick_family(int mode, int d, int k) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-  size_t off_state, off_S, off_F, off_g, off_u, off_partials, total;
-  int max_slots;
+  size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, total;
+  int max_slots, max_groups;
 };
 
 static int device_sm_count() {
@@ -138,6 +139,9 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   w.off_u = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k * d, 256);
   w.max_slots = sms * MAX_BLOCKS_PER_SM + n_layers;
   w.off_partials = o; o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen_max, 256);
+  w.max_groups = w.max_slots / RED_GROUP + n_layers + 2;
+  w.off_gpartials = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups * plen_max, 256);
+  w.off_gtickets = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups, 256);
   w.total = o;
   *out = w;
   return true;
@@ -237,6 +241,8 @@ static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p)
   p->gvec = reinterpret_cast<float*>(ws + wl.off_g);
   p->u = reinterpret_cast<float*>(ws + wl.off_u);
   p->partials = reinterpret_cast<double*>(ws + wl.off_partials);
+  p->gpartials = reinterpret_cast<double*>(ws + wl.off_gpartials);
+  p->gtickets = reinterpret_cast<unsigned int*>(ws + wl.off_gtickets);
   p->st = reinterpret_cast<LayerState*>(ws + wl.off_state);
   p->inv_tau = (float)(1.0 / (double)ctx->tau);
   p->inv_tau_d = 1.0 / (double)ctx->tau;
@@ -413,7 +419,7 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
   const int n_coord = n_layers * k * d;
   const int init_threads = n_coord > n_layers ? n_coord : n_layers;
   idkm_init_forward<<<(init_threads + 255) / 256, 256, 0, ctx->stream>>>(p.st, n_layers, C0, C_out, n_coord, k, d,
-                                                                                     p.inv_tau_d);
+                                                                                     p.inv_tau_d, p.gtickets, wl.max_groups);
   if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
   ++ctx->launches;
   mark(ctx, 1);

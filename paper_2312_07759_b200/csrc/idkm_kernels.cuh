@@ -24,6 +24,8 @@ constexpr float PAD_COORD = 1e18f;   // coordinate of a padding centroid: exp un
 constexpr double S_MIN = 1e-20;      // column sums below this mark a dead cluster
 constexpr float S_MIN_F = 1e-20f;
 constexpr int MAX_BLOCKS_PER_SM = 8;
+// Blocks whose partials one block adds up in the first stage of the cross-block reduction (see finish_layer).
+constexpr int RED_GROUP = 16;
 // When the bounding box of a layer's centroids is smaller than PRECISE_SPAN * tau, all softmax logits of a
 // weight differ by less than PRECISE_SPAN and the centroid update is decided by attention differences far below
 // fp32 resolution (w - c_j rounds away the differences between the c_j).  Such layers step in fp64.
@@ -72,6 +74,8 @@ struct PassParams {
   float* gvec;        // [L][k][d] direct codebook gradient (GRAD writes)
   float* u;           // [L][k][d] adjoint (GRAD initialises, ADJ updates)
   double* partials;   // [(n_blocks + L)][PLEN]
+  double* gpartials;  // [(n_blocks + L) / RED_GROUP + L + 2][PLEN]: sums over groups of RED_GROUP partials
+  unsigned int* gtickets;   // one arrival counter per group, zero at rest
   LayerState* st;
   float inv_tau;      // 1 / tau
   float scale;        // log2(e) / tau
@@ -212,8 +216,12 @@ __device__ __forceinline__ double block_reduce_double(double v, double* scratch 
 }
 __device__ __forceinline__ double block_sum_double(double v, double* scratch) { return block_reduce_double<0>(v, scratch); }
 
-// After a block has written its partial of layer l: take a ticket; the last contributing block adds the
-// layer's partials in slot order (fp64) and applies the epilogue of the pass.  Called by all threads of the block.
+// After a block has written its partial of layer l, the partials are added up in two stages so that no block
+// ever reads more than RED_GROUP + (blocks / RED_GROUP) of them: the contributing blocks form groups of RED_GROUP
+// consecutive blocks; the last block to arrive in a group adds the group's partials in slot order (fp64) into a
+// group partial; the last group to finish adds the group partials in group order and applies the epilogue of the
+// pass.  Grouping and order depend on block indices only, so the result is reproducible.  Layers with at most
+// RED_GROUP contributing blocks skip the first stage.  Called by all threads of the block.
 // smem_raw must hold (PLEN + BLOCK) doubles.
 template <int MODE, int D, int PLEN, int NA>
 __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, unsigned char* smem_raw, int* s_flag) {
@@ -222,24 +230,57 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   const int nb = p.lt.n_blocks;
   __threadfence();
   __syncthreads();
-  // ticket: the last contributing block of this layer reduces all of the layer's partials
   const int first_b = block_of_tile(p.lt.tile_off[l], p.lt.tiles_total, nb);
   const int last_b = block_of_tile(p.lt.tile_off[l + 1] - 1, p.lt.tiles_total, nb);
   const int n_contrib = last_b - first_b + 1;
+  const double* base = p.partials + (size_t)(first_b + l) * PLEN;   // rows the last stage adds
+  int n_terms = n_contrib;
+  if (n_contrib > RED_GROUP) {
+    // ---- first stage: one group of RED_GROUP consecutive slots ----
+    const int g = (b - first_b) / RED_GROUP;
+    const int gsize = (n_contrib - g * RED_GROUP < RED_GROUP) ? n_contrib - g * RED_GROUP : RED_GROUP;
+    // group rows of layer l start at (first slot / RED_GROUP) + l: distinct layers get distinct rows because a
+    // layer with n slots has at most n / RED_GROUP + 1 groups
+    const int grow0 = (first_b + l) / RED_GROUP + l;
+    if (tid == 0) {
+      const unsigned int prev = atomicAdd(&p.gtickets[grow0 + g], 1u);
+      *s_flag = (prev == (unsigned int)(gsize - 1));
+    }
+    __syncthreads();
+    if (!*s_flag) return;
+    __threadfence();
+    const double* gb = base + (size_t)g * RED_GROUP * PLEN;
+    double* gout = p.gpartials + (size_t)(grow0 + g) * PLEN;
+    for (int o = tid; o < PLEN; o += BLOCK) {
+      double v[RED_GROUP];
+#pragma unroll
+      for (int q = 0; q < RED_GROUP; ++q) v[q] = (q < gsize) ? __ldcg(gb + (size_t)q * PLEN + o) : 0.0;
+      double s = 0.0;
+#pragma unroll
+      for (int q = 0; q < RED_GROUP; ++q) s += v[q];
+      gout[o] = s;
+    }
+    if (tid == 0) p.gtickets[grow0 + g] = 0u;
+    __threadfence();
+    __syncthreads();
+    base = p.gpartials + (size_t)grow0 * PLEN;
+    n_terms = (n_contrib + RED_GROUP - 1) / RED_GROUP;
+  }
+  // ---- last stage: the last arrival (block, or group) adds the remaining rows ----
   if (tid == 0) {
     const unsigned int prev = atomicAdd(&p.st[l].ticket, 1u);
-    *s_flag = (prev == (unsigned int)(n_contrib - 1));
+    *s_flag = (prev == (unsigned int)(n_terms - 1));
   }
   __syncthreads();
   if (!*s_flag) return;
   __threadfence();
   double* tot = reinterpret_cast<double*>(smem_raw);   // [PLEN]
   double* scratch = tot + PLEN;                          // [BLOCK]
-  const double* base = p.partials + (size_t)(first_b + l) * PLEN;
   if constexpr (PLEN >= BLOCK) {
     for (int o = tid; o < PLEN; o += BLOCK) {
       double s = 0.0;
-      for (int q = 0; q < n_contrib; ++q) s += __ldcg(base + (size_t)q * PLEN + o);
+#pragma unroll 8
+      for (int q = 0; q < n_terms; ++q) s += __ldcg(base + (size_t)q * PLEN + o);
       tot[o] = s;
     }
     __syncthreads();
@@ -248,7 +289,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
     const int ch = tid / PLEN, o = tid % PLEN;
     double s = 0.0;
     if (ch < NCH)
-      for (int q = ch; q < n_contrib; q += NCH) s += __ldcg(base + (size_t)q * PLEN + o);
+      for (int q = ch; q < n_terms; q += NCH) s += __ldcg(base + (size_t)q * PLEN + o);
     scratch[tid] = s;
     __syncthreads();
     if (tid < PLEN) {

@@ -31,8 +31,10 @@ static NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
 
 // Resets the single layer's state and seeds C_out with the starting centroids.  The scratch keeps
 // whatever the previous call left, so everything the step reads before writing is set here.
-__global__ void idkm_noalloc_init(LayerState* st, const float* C_in, float* C_out, int k, int d, double inv_tau) {
+__global__ void idkm_noalloc_init(LayerState* st, const float* C_in, float* C_out, int k, int d, double inv_tau,
+                                  unsigned int* gtickets, int n_groups) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  for (int o = i; o < n_groups; o += gridDim.x * blockDim.x) gtickets[o] = 0u;
   if (i == 0) {
     LayerState s;
     memset(&s, 0, sizeof(s));
@@ -124,16 +126,23 @@ extern "C" int idkm_step_noalloc(const float* W, int64_t m, int d, const float* 
   rc = noalloc_table(e64, m, nd.sms, &lt64);
   if (rc != IDKM_OK) return rc;
 
-  // layout of the fixed scratch: [state 256 B][partials of whichever step kernel runs]
-  const size_t need32 = 256 + sizeof(double) * (size_t)(p.lt.n_blocks + 1) * e32->plen;
-  const size_t need64 = 256 + sizeof(double) * (size_t)(lt64.n_blocks + 1) * e64->plen;
-  if (need32 > NOALLOC_SCRATCH_BYTES || need64 > NOALLOC_SCRATCH_BYTES) return IDKM_ERR_NOALLOC_TOO_LARGE;
+  // layout of the fixed scratch: [state 256 B][group counters 1 KB][partials][group partials] of whichever step
+  // kernel runs (the two never run for the same layer in one call)
+  const int nb_max = p.lt.n_blocks > lt64.n_blocks ? p.lt.n_blocks : lt64.n_blocks;
+  const int plen_max = e32->plen > e64->plen ? e32->plen : e64->plen;
+  const int n_groups = (nb_max + 1) / RED_GROUP + 3;
+  const size_t off_gt = 256, off_part = off_gt + 1024;
+  const size_t off_gpart = off_part + sizeof(double) * (size_t)(nb_max + 1) * plen_max;
+  const size_t need = off_gpart + sizeof(double) * (size_t)n_groups * plen_max;
+  if (n_groups * sizeof(unsigned int) > 1024 || need > NOALLOC_SCRATCH_BYTES) return IDKM_ERR_NOALLOC_TOO_LARGE;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   p.W = W;
   p.C = C_out;
   p.st = reinterpret_cast<LayerState*>(nd.scratch);
-  p.partials = reinterpret_cast<double*>(nd.scratch + 256);
+  p.partials = reinterpret_cast<double*>(nd.scratch + off_part);
+  p.gpartials = reinterpret_cast<double*>(nd.scratch + off_gpart);
+  p.gtickets = reinterpret_cast<unsigned int*>(nd.scratch + off_gt);
   p.inv_tau = (float)(1.0 / (double)tau);
   p.inv_tau_d = 1.0 / (double)tau;
   p.scale = (float)(1.4426950408889634 / (double)tau);
@@ -145,7 +154,7 @@ extern "C" int idkm_step_noalloc(const float* W, int64_t m, int d, const float* 
   q = p;
   q.lt = lt64;
 
-  idkm_noalloc_init<<<(k * d + 255) / 256, 256, 0, stream>>>(p.st, C_in, C_out, k, d, p.inv_tau_d);
+  idkm_noalloc_init<<<(k * d + 255) / 256, 256, 0, stream>>>(p.st, C_in, C_out, k, d, p.inv_tau_d, p.gtickets, n_groups);
   if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
   if (e32->launch(p, p.lt.n_blocks, stream) != cudaSuccess) return IDKM_ERR_CUDA;
   if (e64->launch(q, q.lt.n_blocks, stream) != cudaSuccess) return IDKM_ERR_CUDA;
