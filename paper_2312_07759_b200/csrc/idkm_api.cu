@@ -225,6 +225,11 @@ static int build_table(idkm_ctx* ctx, int mode, int family, LayerTable* lt) {
   }
   lt->tiles_total = (int)tiles;
   long long nb = (long long)ctx->sms * blocks_per_sm(ctx, mode, ctx->d, family);
+  // Batched loops: layers drop out of a loop at different times (converged, or handed to the other step kernel),
+  // and the blocks that own their tiles return at once.  With more blocks than fit on the GPU at a time the
+  // hardware scheduler backfills the freed slots with blocks of the layers that still run, instead of leaving SMs
+  // idle for the rest of the launch.
+  if (ctx->n_layers > 1 && (mode == STEP || mode == STEP_PRECISE || mode == ADJ)) nb = (long long)ctx->sms * MAX_BLOCKS_PER_SM;
   if (nb > tiles) nb = tiles;
   lt->n_blocks = (int)nb;
   lt->pad = 0;

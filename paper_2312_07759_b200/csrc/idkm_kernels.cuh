@@ -26,6 +26,9 @@ constexpr float S_MIN_F = 1e-20f;
 constexpr int MAX_BLOCKS_PER_SM = 8;
 // Blocks whose partials one block adds up in the first stage of the cross-block reduction (see finish_layer).
 constexpr int RED_GROUP = 16;
+// Up to this many partials one block adds them all: the extra stage costs a few microseconds of latency, which only
+// pays off once the single stage would read hundreds of rows.
+constexpr int RED_SINGLE_MAX = 64;
 // When the bounding box of a layer's centroids is smaller than PRECISE_SPAN * tau, all softmax logits of a
 // weight differ by less than PRECISE_SPAN and the centroid update is decided by attention differences far below
 // fp32 resolution (w - c_j rounds away the differences between the c_j).  Such layers step in fp64.
@@ -221,7 +224,7 @@ __device__ __forceinline__ double block_sum_double(double v, double* scratch) { 
 // consecutive blocks; the last block to arrive in a group adds the group's partials in slot order (fp64) into a
 // group partial; the last group to finish adds the group partials in group order and applies the epilogue of the
 // pass.  Grouping and order depend on block indices only, so the result is reproducible.  Layers with at most
-// RED_GROUP contributing blocks skip the first stage.  Called by all threads of the block.
+// RED_SINGLE_MAX contributing blocks skip the first stage.  Called by all threads of the block.
 // smem_raw must hold (PLEN + BLOCK) doubles.
 template <int MODE, int D, int PLEN, int NA>
 __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, unsigned char* smem_raw, int* s_flag) {
@@ -235,7 +238,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   const int n_contrib = last_b - first_b + 1;
   const double* base = p.partials + (size_t)(first_b + l) * PLEN;   // rows the last stage adds
   int n_terms = n_contrib;
-  if (n_contrib > RED_GROUP) {
+  if (n_contrib > RED_SINGLE_MAX) {
     // ---- first stage: one group of RED_GROUP consecutive slots ----
     const int g = (b - first_b) / RED_GROUP;
     const int gsize = (n_contrib - g * RED_GROUP < RED_GROUP) ? n_contrib - g * RED_GROUP : RED_GROUP;
@@ -974,6 +977,9 @@ struct PreciseCfg {
   static constexpr int PLEN = KP * NA;
   static constexpr int WPG = (LPW == 1) ? 4 : 16;   // small tiles in the thread-per-weight layouts spread small layers
   static constexpr int TILE = (BLOCK / LPW) * WPG;
+  // small codebooks in the thread-per-weight layout: four resident blocks per SM (64 registers) hide the latency of
+  // the dependent fp64 chains better than two blocks with more rows in flight each
+  static constexpr int MIN_BLOCKS = (LPW == 1 && KPL * (D + 1) <= 8) ? 4 : 1;
 };
 
 __device__ __forceinline__ double exp_small(double y) {   // |y| <= PRECISE_SPAN: truncation error y^7/5040 < 8e-13
@@ -1000,7 +1006,8 @@ __device__ __forceinline__ double group_min_d(double v) {
 }
 
 template <int D, int KPL, int LPW>
-__global__ void __launch_bounds__(BLOCK) idkm_step_precise(const __grid_constant__ PassParams p) {
+__global__ void __launch_bounds__(BLOCK, PreciseCfg<D, KPL, LPW>::MIN_BLOCKS)
+idkm_step_precise(const __grid_constant__ PassParams p) {
   using Cfg = PreciseCfg<D, KPL, LPW>;
   constexpr int NA = Cfg::NA;
   constexpr int PLEN = Cfg::PLEN;
@@ -1087,7 +1094,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_step_precise(const __grid_constant
     // its own WPG consecutive rows
     const long long tb = (long long)(tile - p.lt.tile_off[layer]) * TILE;
     // all rows of the trip are fetched first (thread-per-weight layouts: 4 loads in flight per thread)
-    constexpr int QB = (LPW == 1) ? WPG : 2;   // rows per fully unrolled batch
+    constexpr int QB = (LPW == 1 && Cfg::MIN_BLOCKS == 1) ? WPG : 2;   // rows per fully unrolled batch
 #pragma unroll 1
     for (int q0 = 0; q0 < WPG; q0 += QB) {
       float wf[QB][D];
