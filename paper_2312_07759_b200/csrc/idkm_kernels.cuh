@@ -14,6 +14,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <type_traits>
 
 namespace idkm {
 
@@ -982,26 +983,32 @@ struct PreciseCfg {
   static constexpr int MIN_BLOCKS = (LPW == 1 && KPL * (D + 1) <= 8) ? 4 : 1;
 };
 
-__device__ __forceinline__ double exp_small(double y) {   // |y| <= PRECISE_SPAN: truncation error y^7/5040 < 8e-13
-  double s = 1.0 / 720.0;
-  s = fma(s, y, 1.0 / 120.0);
-  s = fma(s, y, 1.0 / 24.0);
-  s = fma(s, y, 1.0 / 6.0);
-  s = fma(s, y, 0.5);
-  s = fma(s, y, 1.0);
-  return fma(s, y, 1.0);
+// exp(z / tau) for |z / tau| <= PRECISE_SPAN by the Taylor series to the sixth power (truncation error
+// y^7/5040 < 8e-13 relative), with 1 / tau folded into the coefficients ec[n] = (1/tau)^(n+1) / (n+1)!: six fused
+// multiply-adds and no separate scaling.  (1/tau)^6 is finite for every positive float tau.
+__device__ __forceinline__ void exp_scaled_coeffs(double inv_tau, double (&ec)[6]) {
+  const double f[6] = {1.0, 0.5, 1.0 / 6.0, 1.0 / 24.0, 1.0 / 120.0, 1.0 / 720.0};
+  double pw = inv_tau;
+#pragma unroll
+  for (int n = 0; n < 6; ++n) {
+    ec[n] = pw * f[n];
+    pw *= inv_tau;
+  }
+}
+__device__ __forceinline__ double exp_scaled(double z, const double (&ec)[6]) {
+  double s = ec[5];
+  s = fma(s, z, ec[4]);
+  s = fma(s, z, ec[3]);
+  s = fma(s, z, ec[2]);
+  s = fma(s, z, ec[1]);
+  s = fma(s, z, ec[0]);
+  return fma(s, z, 1.0);
 }
 
 template <int LPW>
 __device__ __forceinline__ double group_sum_d(double v) {
 #pragma unroll
   for (int o = LPW / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-template <int LPW>
-__device__ __forceinline__ double group_min_d(double v) {
-#pragma unroll
-  for (int o = LPW / 2; o > 0; o >>= 1) v = fmin(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
 
@@ -1034,6 +1041,8 @@ idkm_step_precise(const __grid_constant__ PassParams p) {
 
   double c[KPL][D];
   double acc[KPL][NA];
+  double ec[6];
+  exp_scaled_coeffs(p.inv_tau_d, ec);
   int layer = 0;
   while (p.lt.tile_off[layer + 1] <= t_lo) ++layer;
   int cur_layer = -1;
@@ -1095,63 +1104,73 @@ idkm_step_precise(const __grid_constant__ PassParams p) {
     const long long tb = (long long)(tile - p.lt.tile_off[layer]) * TILE;
     // all rows of the trip are fetched first (thread-per-weight layouts: 4 loads in flight per thread)
     constexpr int QB = (LPW == 1 && Cfg::MIN_BLOCKS == 1) ? WPG : 2;   // rows per fully unrolled batch
+    // one body for codebooks that fill every centroid slot of the layout (no per-centroid validity tests) and one
+    // for padded codebooks
+    auto rows_of_tile = [&](auto full_tag) {
+      constexpr bool FULL = decltype(full_tag)::value;
 #pragma unroll 1
-    for (int q0 = 0; q0 < WPG; q0 += QB) {
-      float wf[QB][D];
-      bool okq[QB];
+      for (int q0 = 0; q0 < WPG; q0 += QB) {
+        float wf[QB][D];
+        bool okq[QB];
 #pragma unroll
-      for (int qq = 0; qq < QB; ++qq) {
-        const int q = q0 + qq;
-        const long long loc = (LPW == 1) ? tb + (long long)q * BLOCK + grp : tb + (long long)grp * WPG + q;
-        okq[qq] = (loc < rows);
-        const long long grow = row0 + (okq[qq] ? loc : 0);
+        for (int qq = 0; qq < QB; ++qq) {
+          const int q = q0 + qq;
+          const long long loc = (LPW == 1) ? tb + (long long)q * BLOCK + grp : tb + (long long)grp * WPG + q;
+          okq[qq] = (loc < rows);
+          const long long grow = row0 + (okq[qq] ? loc : 0);
 #pragma unroll
-        for (int a = 0; a < D; ++a) wf[qq][a] = __ldg(p.W + grow * D + a);
-      }
+          for (int a = 0; a < D; ++a) wf[qq][a] = __ldg(p.W + grow * D + a);
+        }
 #pragma unroll
-      for (int qq = 0; qq < QB; ++qq) {
-        double w[D];
+        for (int qq = 0; qq < QB; ++qq) {
+          double w[D];
 #pragma unroll
-        for (int a = 0; a < D; ++a) w[a] = (double)wf[qq][a];
-        double dist[KPL];
-        double lmin = 1e300;
+          for (int a = 0; a < D; ++a) w[a] = (double)wf[qq][a];
+          double dist[KPL];
 #pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          double sq = 0.0;
+          for (int t = 0; t < KPL; ++t) {
+            double sq = 0.0;
 #pragma unroll
-          for (int a = 0; a < D; ++a) {
-            const double df = w[a] - c[t][a];
-            sq = (D == 1) ? fabs(df) : fma(df, df, sq);
+            for (int a = 0; a < D; ++a) {
+              const double df = w[a] - c[t][a];
+              sq = (D == 1) ? fabs(df) : fma(df, df, sq);
+            }
+            dist[t] = (D == 1) ? sq : sqrt(sq);
           }
-          dist[t] = (D == 1) ? sq : sqrt(sq);
-          if (gl * KPL + t < k) lmin = fmin(lmin, dist[t]);
-        }
-        const double gmin = group_min_d<LPW>(lmin);
-        double e[KPL];
-        double lsum = 0.0;
+          // Softmax reference: the distance to centroid 0 instead of the row minimum.  All centroids of a `precise`
+          // layer lie within PRECISE_SPAN * tau of each other, so by the triangle inequality every
+          // (reference - D_ij) / tau stays within +-PRECISE_SPAN, which is all exp_scaled needs.
+          double ref = dist[0];
+          if constexpr (LPW > 1) ref = __shfl_sync(0xffffffffu, ref, lane - gl);
+          double e[KPL];
+          double lsum = 0.0;
 #pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          e[t] = (gl * KPL + t < k) ? exp_small((gmin - dist[t]) * p.inv_tau_d) : 0.0;
-          lsum += e[t];
-        }
-        const double gsum = group_sum_d<LPW>(lsum);
-        // reciprocal of the row sum (1 <= gsum <= k): fp32 seed and two Newton steps in fp64 (error ~1e-28 relative
-        // to the seed's 1e-7 squared twice), cheaper than a double division
-        double r = (double)rcp_approx((float)gsum);
-        r = r * (2.0 - gsum * r);
-        r = r * (2.0 - gsum * r);
-        if (!okq[qq]) r = 0.0;
-        double rw[D];
+          for (int t = 0; t < KPL; ++t) {
+            const double ev = exp_scaled(ref - dist[t], ec);
+            e[t] = (FULL || gl * KPL + t < k) ? ev : 0.0;
+            lsum += e[t];
+          }
+          const double gsum = group_sum_d<LPW>(lsum);
+          // reciprocal of the row sum (about k): fp32 seed and two Newton steps in fp64 (error ~1e-28 relative
+          // to the seed's 1e-7 squared twice), cheaper than a double division
+          double r = (double)rcp_approx((float)gsum);
+          r = r * (2.0 - gsum * r);
+          r = r * (2.0 - gsum * r);
+          if (!okq[qq]) r = 0.0;
+          double rw[D];
 #pragma unroll
-        for (int a = 0; a < D; ++a) rw[a] = r * w[a];
+          for (int a = 0; a < D; ++a) rw[a] = r * w[a];
 #pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          acc[t][0] = fma(e[t], r, acc[t][0]);
+          for (int t = 0; t < KPL; ++t) {
+            acc[t][0] = fma(e[t], r, acc[t][0]);
 #pragma unroll
-          for (int a = 0; a < D; ++a) acc[t][1 + a] = fma(e[t], rw[a], acc[t][1 + a]);
+            for (int a = 0; a < D; ++a) acc[t][1 + a] = fma(e[t], rw[a], acc[t][1 + a]);
+          }
         }
       }
-    }
+    };
+    if (k == Cfg::KP) rows_of_tile(std::true_type{});
+    else rows_of_tile(std::false_type{});
   }
   grid_release_dependents();
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
