@@ -689,13 +689,14 @@ idkm_pass(const __grid_constant__ PassParams p) {
       }
       const float zbar = group_sum<LPW>((lzp[0] + lzp[1]) + (lzp[2] + lzp[3])) * r;
       const float rt = r * p.inv_tau;
+      const float nzr = -zbar * rt;
       float dwl[D];
 #pragma unroll
       for (int a = 0; a < D; ++a) dwl[a] = 0.f;
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
         const float at = e[t] * r;                    // A_ij
-        float et = e[t] * rt * (z[t] - zbar);         // e_ij(z) / tau
+        float et = e[t] * fmaf(z[t], rt, nzr);        // e_ij(z) / tau = A_ij (z_ij - zbar_i) / tau
         if constexpr (D > 1) et *= rs[t];             // ... / D_ij, so that et * (w - c) = e_ij(z) n_ij / tau
 #pragma unroll
         for (int a = 0; a < D; ++a) {
