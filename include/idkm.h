@@ -54,6 +54,7 @@ extern "C" {
 #define IDKM_ERR_CUDA (-8)       /* a CUDA runtime call failed                                  */
 #define IDKM_ERR_NONFINITE (-9)  /* device: NaN/Inf met in W, C or the sums                     */
 #define IDKM_ERR_NOALLOC_TOO_LARGE (-11) /* idkm_step_noalloc: the problem needs more than the built-in scratch */
+#define IDKM_ERR_TIMEOUT (-12)   /* device: a bounded grid-wide wait of the one-launch forward loop ran out  */
 #define IDKM_ERR_DIVERGED (-10)  /* device: adjoint iteration produced non-finite values or its
                                     residual grew 10 steps running (Section 4.2: retry with a
                                     smaller alpha)                                              */
@@ -206,6 +207,18 @@ int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
  * measurement.  Synchronises cuda_stream.  Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_CUDA.
  */
 int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_per_s, void* cuda_stream);
+
+/*
+ * How the forward loop (Algorithm 1) is launched.  0 (default): a single layer with k <= 8 and at most about 2.4
+ * million rows (32 rows per thread of the co-resident grid) runs the WHOLE loop in one cooperative launch: per
+ * iteration every block publishes one fp64 partial, all blocks meet at a grid-wide barrier, and every block then
+ * adds the partials in the same order and takes the M-step itself, so only the partials cross L2 inside the loop;
+ * the loop leaves at the iteration whose stop test passes.  Everything else (batched layers, larger layers or
+ * codebooks, max_iter < 2) takes one launch per iteration.  Every barrier wait is bounded (about a second): if one
+ * runs out the kernel returns and the layer's status is IDKM_ERR_TIMEOUT.  1: always one launch per iteration.
+ * Both run the same iteration; results differ only by the order of the cross-block sums.
+ */
+int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 
 /* Number of kernels this ctx has launched since idkm_create (for accounting in benchmarks). */
 int64_t idkm_launch_count(const idkm_ctx* ctx);

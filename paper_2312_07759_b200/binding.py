@@ -62,6 +62,8 @@ lib.idkm_step_noalloc.argtypes = [_fp, C.c_int64, C.c_int, _fp, C.c_int, C.c_flo
 lib.idkm_step_noalloc.restype = C.c_int
 lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
 lib.idkm_set_adjoint_method.restype = C.c_int
+lib.idkm_set_forward_loop.argtypes = [_vp, C.c_int]
+lib.idkm_set_forward_loop.restype = C.c_int
 lib.idkm_launch_count.argtypes = [_vp]
 lib.idkm_launch_count.restype = C.c_int64
 lib.idkm_measure_pipe_rates.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), _vp]
@@ -237,6 +239,10 @@ class Context:
     def set_adjoint_method(self, method: int) -> None:
         """0: explicit Jacobian for k*d <= 8 (default); 1: always one fused pass per adjoint step."""
         _check(lib.idkm_set_adjoint_method(self._h, int(method)))
+
+    def set_forward_loop(self, method: int) -> None:
+        """0: small layers run the whole forward loop in one cooperative launch (default); 1: a launch per iteration."""
+        _check(lib.idkm_set_forward_loop(self._h, int(method)))
 
     def set_timing(self, enable: bool = True) -> None:
         _check(lib.idkm_set_timing(self._h, 1 if enable else 0))

@@ -21,12 +21,14 @@ extern const KernelEntry k_table_adj[3][N_FAMILY];
 extern const KernelEntry k_table_scatter[3][N_FAMILY];
 extern const KernelEntry k_table_step_precise[3][N_FAMILY];
 extern const KernelEntry k_table_jacobian[3][N_FAMILY];
+extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
-                                  double inv_tau, unsigned int* gtickets, int n_groups) {
+                                  double inv_tau, unsigned int* gtickets, int n_groups, unsigned int* sync) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   for (int o = i; o < n_groups; o += gridDim.x * blockDim.x) gtickets[o] = 0u;
+  if (i < 4) sync[i] = 0u;
   if (i < n_layers) {
     LayerState s;
     s.fwd_done = 0; s.fwd_iters = 0; s.fwd_res = 0.f; s.dead = 0;
@@ -106,7 +108,7 @@ int pick_family(int mode, int d, int k) {
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct WorkspaceLayout {
-  size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, total;
+  size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, off_sync, total;
   int max_slots, max_groups;
 };
 
@@ -142,6 +144,7 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   w.max_groups = w.max_slots / RED_GROUP + n_layers + 2;
   w.off_gpartials = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups * plen_max, 256);
   w.off_gtickets = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups, 256);
+  w.off_sync = o;      o = align_up(o + 4 * sizeof(unsigned int), 256);   // barrier words of the single-launch loop
   w.total = o;
   *out = w;
   return true;
@@ -174,6 +177,8 @@ struct idkm_ctx {
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
+  int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never
+  int small_blocks[3][N_SMALL_FAMILY];   // cached co-resident grid of the single-launch loop kernels (0 = not queried)
   // bounded run-ahead of the tolerance-mode loops: a pinned host word the device sets when all layers are done
   int* h_flag;
   int* d_flag;
@@ -315,6 +320,62 @@ static int launch_step_loop(idkm_ctx* ctx, PassParams* p, int repeat) {
   return IDKM_OK;
 }
 
+// The single-launch loop takes a single layer with k <= 8 whose rows fit SMALL_ROWS_PER_THREAD per thread of the
+// co-resident grid (so that a thread's fp32 sums stay short, as in the tiled passes) -- about 2.4 million rows on a
+// 148-SM part.  Blocks get at least SMALL_MIN_ROWS_PER_THREAD rows per thread: tiny layers use few blocks, which keeps
+// the cross-block sum short.
+constexpr int SMALL_ROWS_PER_THREAD = 32;
+constexpr int SMALL_MIN_ROWS_PER_THREAD = 4;
+constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM clock ticks per barrier wait
+
+// Returns IDKM_OK after queueing the loop, 1 if this problem should take the launch-per-iteration path.
+static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p, int max_iter) {
+  static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
+  if (env_off || ctx->forward_loop != 0 || ctx->n_layers != 1 || max_iter < 2) return 1;
+  const int di = d_index(ctx->d);
+  int f = -1;
+  for (int q = 0; q < N_SMALL_FAMILY; ++q)
+    if (k_table_small[di][q].kpl >= ctx->k) { f = q; break; }
+  if (f < 0) return 1;
+  const SmallLoopEntry* se = &k_table_small[di][f];
+  int& nb = ctx->small_blocks[di][f];
+  if (nb == 0) {
+    int coop = 0, per_sm = 0;
+    nb = -1;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, se->func, BLOCK, 0) == cudaSuccess && per_sm >= 1)
+      nb = ctx->sms * (per_sm > 2 ? 2 : per_sm);
+    (void)cudaGetLastError();
+  }
+  if (nb <= 0) return 1;
+  const long long m = ctx->m_total;
+  if (m > (long long)SMALL_ROWS_PER_THREAD * nb * BLOCK) return 1;
+  long long grid = (m + (long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK - 1) / ((long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK);
+  if (grid > nb) grid = nb;
+  if (grid < 1) grid = 1;
+  if (2 * grid > wl.max_slots) return 1;   // the two partial buffers live in the partial-slot region
+  SmallLoopParams sp;
+  memset(&sp, 0, sizeof(sp));
+  sp.W = ctx->W;
+  sp.m = m;
+  sp.C = ctx->C;
+  sp.st = p.st;
+  sp.partials = p.partials;
+  sp.sync = reinterpret_cast<unsigned int*>(static_cast<char*>(ctx->workspace) + wl.off_sync);
+  sp.k = ctx->k;
+  sp.scale = p.scale;
+  sp.tol = p.tol;
+  sp.inv_tau_d = p.inv_tau_d;
+  sp.max_iter = max_iter;
+  sp.spin_limit = SMALL_SPIN_LIMIT;
+  if (se->launch(sp, (int)grid, ctx->stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 1;   // nothing was queued: take the launch-per-iteration path
+  }
+  ++ctx->launches;
+  return IDKM_OK;
+}
+
 static int launch_pass(idkm_ctx* ctx, int mode, PassParams* p, int repeat) {
   const int f = pick_family(mode, ctx->d, ctx->k);
   const KernelEntry* e = kernel_entry(mode, ctx->d, f);
@@ -424,12 +485,14 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
   const int n_coord = n_layers * k * d;
   const int init_threads = n_coord > n_layers ? n_coord : n_layers;
   idkm_init_forward<<<(init_threads + 255) / 256, 256, 0, ctx->stream>>>(p.st, n_layers, C0, C_out, n_coord, k, d,
-                                                                                     p.inv_tau_d, p.gtickets, wl.max_groups);
+                                                                                     p.inv_tau_d, p.gtickets, wl.max_groups,
+                                                                                     reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + wl.off_sync));
   if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
   ++ctx->launches;
   mark(ctx, 1);
 
-  int rc = launch_step_loop(ctx, &p, max_iter);
+  int rc = try_small_loop(ctx, wl, p, max_iter);
+  if (rc == 1) rc = launch_step_loop(ctx, &p, max_iter);
   if (rc != IDKM_OK) return rc;
   mark(ctx, 2);
   p.Wq = Wq_out;
@@ -615,6 +678,13 @@ int idkm_set_adjoint_method(idkm_ctx* ctx, int method) {
   return IDKM_OK;
 }
 
+int idkm_set_forward_loop(idkm_ctx* ctx, int method) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (method != 0 && method != 1) return IDKM_ERR_PARAM;
+  ctx->forward_loop = method;
+  return IDKM_OK;
+}
+
 int64_t idkm_launch_count(const idkm_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 const char* idkm_status_string(int status) {
@@ -632,6 +702,7 @@ const char* idkm_status_string(int status) {
     case IDKM_ERR_NONFINITE: return "non-finite value met on the device";
     case IDKM_ERR_DIVERGED: return "adjoint iteration diverged";
     case IDKM_ERR_NOALLOC_TOO_LARGE: return "problem needs more than the library's built-in scratch";
+    case IDKM_ERR_TIMEOUT: return "a grid-wide wait of the single-launch forward loop ran out";
   }
   return "unknown status";
 }

@@ -39,7 +39,7 @@ enum Mode { STEP = 0, FINAL = 1, GRAD = 2, ADJ = 3, SCATTER = 4, STEP_PRECISE = 
 constexpr int N_MODES = 7;
 
 // status values mirrored from idkm.h (device side needs only these)
-constexpr int ST_OK = 0, ST_MAXITER = 1, ST_NONFINITE = -9, ST_DIVERGED = -10;
+constexpr int ST_OK = 0, ST_MAXITER = 1, ST_NONFINITE = -9, ST_DIVERGED = -10, ST_TIMEOUT = -12;
 
 struct LayerState {   // 64 bytes, one per layer, in the workspace
   int fwd_done, fwd_iters;
@@ -1447,6 +1447,28 @@ struct KernelEntry {
   int kpl, lpw, tile, plen;
   int dyn_smem;   // dynamic shared memory the launch asks for (bytes)
 };
+// Single-launch forward loop for one small layer (idkm_small_loop.cu): k <= 2, 4, 8 centroids per thread.
+struct SmallLoopParams {
+  const float* W;
+  long long m;
+  float* C;              // [k][d]: starting centroids in, returned centroids out
+  LayerState* st;        // the layer's state: `precise` is read at the start, the outcome written at the end
+  double* partials;      // [2][grid][k_pad (d+1)] fp64 block partials, alternating by iteration
+  unsigned int* sync;    // [0] barrier arrivals (only grows), [1] error word; both zero before the launch
+  int k;
+  float scale;           // log2(e) / tau
+  float tol;
+  double inv_tau_d;
+  int max_iter;
+  long long spin_limit;  // clock64() ticks a block waits at a barrier before it gives up
+};
+typedef cudaError_t (*SmallLaunchFn)(const SmallLoopParams& sp, int grid, cudaStream_t stream);
+struct SmallLoopEntry {
+  SmallLaunchFn launch;
+  const void* func;
+  int kpl, plen;
+};
+constexpr int N_SMALL_FAMILY = 3;
 // family index f: 0..7 -> supports k <= kpl*lpw
 constexpr int N_FAMILY = 9;
 const KernelEntry* kernel_entry(int mode, int d, int family);

@@ -1,0 +1,317 @@
+// Algorithm 1's whole loop in ONE cooperative launch, for a single small layer (k <= 8, a few million weights at most).
+//
+// There one iteration is a few microseconds of arithmetic, and a launch per iteration -- with its chain of dependent
+// trips to L2 (partials, ticket, totals, centroids, state) -- costs more than the arithmetic.  Here all blocks are
+// co-resident; per iteration each block adds up its rows, publishes one fp64 partial, waits at a grid-wide barrier
+// (one counter that only grows), and then EVERY block adds all partials in the same fixed order and takes the M-step
+// itself: centroids, iteration count, residual and stop flag live in registers / shared memory of every block and are
+// bit-identical everywhere, so nothing but the partials crosses L2 inside the loop.  W is read through the read-only
+// path and stays in L1 from the second iteration on.  Block 0 writes the centroids and the layer state once, at the end.
+#include "idkm_kernels.cuh"
+
+namespace idkm {
+
+template <int D, int KPL>
+struct SmallCfg {
+  static constexpr int NA = D + 1;
+  static constexpr int PLEN = KPL * NA;
+  static constexpr int CH = BLOCK / PLEN;          // chunks of partial rows added in parallel in the second level
+  static constexpr int KD = KPL * D;
+};
+
+// Bounded wait until the arrival counter has reached `target`.  Returns false if the wait ran out or another block
+// raised the error word.
+__device__ __forceinline__ bool small_barrier(unsigned int* sync, unsigned int target, long long spin_limit, int* s_ok) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    volatile unsigned int* vs = sync;
+    int ok = 1;
+    __threadfence();
+    atomicAdd(&sync[0], 1u);
+    const long long t0 = clock64();
+    while ((int)(vs[0] - target) < 0) {
+      if (vs[1] != 0u || clock64() - t0 > spin_limit) {
+        atomicExch(&sync[1], 1u);
+        ok = 0;
+        break;
+      }
+    }
+    if (vs[1] != 0u) ok = 0;
+    __threadfence();
+    *s_ok = ok;
+  }
+  __syncthreads();
+  return *s_ok != 0;
+}
+
+template <int D, int KPL>
+__global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constant__ SmallLoopParams sp) {
+  using Cfg = SmallCfg<D, KPL>;
+  constexpr int NA = Cfg::NA, PLEN = Cfg::PLEN, CH = Cfg::CH, KD = Cfg::KD;
+  __shared__ float red[NWARP][PLEN];
+  __shared__ double redd[NWARP][PLEN];
+  __shared__ double chunk[CH][PLEN];
+  __shared__ double tot[PLEN];
+  __shared__ float c_sm[KD > 0 ? KD : 1];   // the current centroids (every block holds the same values)
+  __shared__ double s_res[4];       // residual, dead, bad, box2
+  __shared__ int s_ok;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int b = blockIdx.x, G = gridDim.x;
+  const int k = sp.k;
+  const long long m = sp.m;
+
+  // uniform loop state (identical in every thread of every block)
+  int iters = 0, done = 0, status = ST_OK, dead_n = 0;
+  int precise = sp.st[0].precise;
+  float res_f = 0.f;
+  if (tid < k * D) c_sm[tid] = sp.C[tid];
+  __syncthreads();
+  float c[KPL][D];
+#pragma unroll
+  for (int t = 0; t < KPL; ++t)
+#pragma unroll
+    for (int a = 0; a < D; ++a) c[t][a] = (t < k) ? c_sm[t * D + a] : PAD_COORD;
+  double ec[6];
+  exp_scaled_coeffs(sp.inv_tau_d, ec);
+  bool ok = true;
+
+  for (int it = 0; it < sp.max_iter && !done; ++it) {
+    // ---- this block's rows and its partial (fixed order: lanes by shuffle tree, warps in index order) ----
+    double* mine = sp.partials + ((size_t)(it & 1) * G + b) * PLEN;
+    auto load_row = [&](long long r, float (&w)[D]) {
+      if constexpr (D == 4) {
+        const float4 x = __ldg(reinterpret_cast<const float4*>(sp.W) + r);
+        w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
+      } else if constexpr (D == 2) {
+        const float2 x = __ldg(reinterpret_cast<const float2*>(sp.W) + r);
+        w[0] = x.x; w[1] = x.y;
+      } else {
+        w[0] = __ldg(sp.W + r);
+      }
+    };
+    if (!precise) {
+      // fp32 rows: the arithmetic of the fused forward step (Algorithm 1, steps 3-5)
+      float acc[KPL][NA];
+#pragma unroll
+      for (int t = 0; t < KPL; ++t)
+#pragma unroll
+        for (int a = 0; a < NA; ++a) acc[t][a] = 0.f;
+      for (long long r = (long long)b * BLOCK + tid; r < m; r += (long long)G * BLOCK) {
+        float w[D];
+        load_row(r, w);
+        float dist[KPL], e[KPL];
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          if constexpr (D == 1) {
+            dist[t] = fabsf(w[0] - c[t][0]);
+          } else {
+            float sq = 0.f;
+#pragma unroll
+            for (int a = 0; a < D; ++a) {
+              const float df = w[a] - c[t][a];
+              sq = fmaf(df, df, sq);
+            }
+            dist[t] = sqrt_approx(sq);
+          }
+        }
+        const float mref = tree_reduce<KPL, 1>(dist) * sp.scale;
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) e[t] = ex2_approx(fmaf(-sp.scale, dist[t], mref));
+        const float rr = rcp_approx(tree_reduce<KPL, 0>(e));
+        float rw[D];
+#pragma unroll
+        for (int a = 0; a < D; ++a) rw[a] = rr * w[a];
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          acc[t][0] = fmaf(e[t], rr, acc[t][0]);
+#pragma unroll
+          for (int a = 0; a < D; ++a) acc[t][1 + a] = fmaf(e[t], rw[a], acc[t][1 + a]);
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < KPL; ++t)
+#pragma unroll
+        for (int a = 0; a < NA; ++a) {
+          float v = acc[t][a];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == 0) red[warp][t * NA + a] = v;
+        }
+      __syncthreads();
+      if (tid < PLEN) {
+        double s = 0.0;
+#pragma unroll
+        for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
+        __stcg(mine + tid, s);
+      }
+    } else {
+      // fp64 rows for a collapsing layer: fp64 distances, a short Taylor exp around the distance to centroid 0 (all
+      // centroids lie within PRECISE_SPAN * tau of each other), fp64 sums
+      double accd[KPL][NA];
+#pragma unroll
+      for (int t = 0; t < KPL; ++t)
+#pragma unroll
+        for (int a = 0; a < NA; ++a) accd[t][a] = 0.0;
+      for (long long r = (long long)b * BLOCK + tid; r < m; r += (long long)G * BLOCK) {
+        float w[D];
+        load_row(r, w);
+        double wd[D], dist[KPL], e[KPL];
+#pragma unroll
+        for (int a = 0; a < D; ++a) wd[a] = (double)w[a];
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          double sq = 0.0;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const double df = wd[a] - (double)c[t][a];
+            sq = (D == 1) ? fabs(df) : fma(df, df, sq);
+          }
+          dist[t] = (D == 1) ? sq : sqrt(sq);
+        }
+        double lsum = 0.0;
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          e[t] = (t < k) ? exp_scaled(dist[0] - dist[t], ec) : 0.0;
+          lsum += e[t];
+        }
+        double rr = (double)rcp_approx((float)lsum);
+        rr = rr * (2.0 - lsum * rr);
+        rr = rr * (2.0 - lsum * rr);
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          accd[t][0] = fma(e[t], rr, accd[t][0]);
+#pragma unroll
+          for (int a = 0; a < D; ++a) accd[t][1 + a] = fma(e[t], rr * wd[a], accd[t][1 + a]);
+        }
+      }
+#pragma unroll
+      for (int t = 0; t < KPL; ++t)
+#pragma unroll
+        for (int a = 0; a < NA; ++a) {
+          double v = accd[t][a];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == 0) redd[warp][t * NA + a] = v;
+        }
+      __syncthreads();
+      if (tid < PLEN) {
+        double s = 0.0;
+#pragma unroll
+        for (int wv = 0; wv < NWARP; ++wv) s += redd[wv][tid];
+        __stcg(mine + tid, s);
+      }
+    }
+    // ---- everyone has published: grid-wide barrier ----
+    ok = small_barrier(sp.sync, (unsigned int)(it + 1) * (unsigned int)G, sp.spin_limit, &s_ok);
+    if (!ok) break;
+    // ---- every block adds all partials in the same order ----
+    {
+      const double* base = sp.partials + (size_t)(it & 1) * G * PLEN;
+      const int ch = tid / PLEN, o = tid % PLEN;
+      if (ch < CH) {
+        double s = 0.0;
+        for (int q = ch; q < G; q += CH) s += __ldcg(base + (size_t)q * PLEN + o);
+        chunk[ch][o] = s;
+      }
+      __syncthreads();
+      if (tid < PLEN) {
+        double s = 0.0;
+#pragma unroll 1
+        for (int q = 0; q < CH; ++q) s += chunk[q][tid];
+        tot[tid] = s;
+      }
+      __syncthreads();
+    }
+    // ---- M-step by the first warp: lane (j, a) owns coordinate a of centroid j ----
+    if (warp == 0) {
+      const int j = lane / D, a = lane % D;
+      (void)a;
+      const bool own = (lane < k * D);
+      double num = 0.0, den = 0.0, bad = 0.0, dead = 0.0, cq = 0.0;
+      if (own) {
+        const double s = tot[j * NA];
+        const bool alive = (s >= S_MIN);
+        const double cold = (double)c_sm[lane];
+        const double cnew = alive ? tot[j * NA + 1 + a] / s : cold;
+        if (!alive && a == 0) dead = 1.0;
+        if (!(s == s) || s > 1e300 || !(cnew == cnew) || fabs(cnew) > 1e300) bad = 1.0;
+        num = (cnew - cold) * (cnew - cold);
+        den = cnew * cnew;
+        cq = (double)(float)cnew;
+        c_sm[lane] = (float)cnew;
+      }
+      double lo = own ? cq : 1e300, hi = own ? cq : -1e300;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        num += __shfl_xor_sync(0xffffffffu, num, o);
+        den += __shfl_xor_sync(0xffffffffu, den, o);
+        bad += __shfl_xor_sync(0xffffffffu, bad, o);
+        dead += __shfl_xor_sync(0xffffffffu, dead, o);
+      }
+      // bounding box per coordinate: lanes with equal a differ by multiples of D
+#pragma unroll
+      for (int o = 16; o >= D; o >>= 1) {
+        lo = fmin(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+      }
+      double ext = (lane < D) ? (hi - lo) * (hi - lo) : 0.0;
+#pragma unroll
+      for (int o = D / 2; o > 0; o >>= 1) ext += __shfl_xor_sync(0xffffffffu, ext, o);
+      if (lane == 0) {
+        double dn = sqrt(den);
+        if (dn < 1e-300) dn = 1e-300;
+        s_res[0] = sqrt(num) / dn;
+        s_res[1] = dead;
+        s_res[2] = bad;
+        s_res[3] = ext;
+      }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < KPL; ++t)
+#pragma unroll
+      for (int a = 0; a < D; ++a) c[t][a] = (t < k) ? c_sm[t * D + a] : PAD_COORD;
+    iters = it + 1;
+    res_f = (float)s_res[0];
+    dead_n = (int)s_res[1];
+    precise = (sqrt(s_res[3]) * sp.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
+    if (s_res[2] > 0.0) {
+      status = ST_NONFINITE;
+      done = 1;
+    } else if (sp.tol > 0.f && res_f < sp.tol) {
+      done = 1;
+      status = ST_OK;
+    } else if (sp.tol > 0.f && iters >= sp.max_iter) {
+      status = ST_MAXITER;
+    }
+    __syncthreads();
+  }
+
+  if (b == 0) {
+    if (tid < k * D) sp.C[tid] = c_sm[tid];
+    if (tid == 0) {
+      LayerState* st = sp.st;
+      st->fwd_iters = iters;
+      st->fwd_res = res_f;
+      st->dead = dead_n;
+      st->fwd_done = done;
+      st->precise = precise;
+      st->status = ok ? status : ST_TIMEOUT;
+      st->ticket = 0u;
+    }
+  }
+}
+
+template <int D, int KPL>
+static cudaError_t launch_small(const SmallLoopParams& sp, int grid, cudaStream_t stream) {
+  void* args[1] = {const_cast<SmallLoopParams*>(&sp)};
+  // cooperative launch: refused (instead of hanging at the first barrier) if the grid cannot be co-resident
+  return cudaLaunchCooperativeKernel((const void*)&idkm_small_loop<D, KPL>, dim3((unsigned)grid, 1, 1),
+                                     dim3(BLOCK, 1, 1), args, 0, stream);
+}
+#define IDKM_SMALL_ENTRY(D, KPL) { &launch_small<D, KPL>, (const void*)&idkm_small_loop<D, KPL>, KPL, SmallCfg<D, KPL>::PLEN }
+#define IDKM_SMALL_ROW(D) { IDKM_SMALL_ENTRY(D, 2), IDKM_SMALL_ENTRY(D, 4), IDKM_SMALL_ENTRY(D, 8) }
+extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY] = {IDKM_SMALL_ROW(1), IDKM_SMALL_ROW(2), IDKM_SMALL_ROW(4)};
+
+}  // namespace idkm

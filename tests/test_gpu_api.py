@@ -134,3 +134,38 @@ def test_pipe_rate_microbenchmarks():
     assert 0.60 < fp32 / (sms * 128 * clk_hz) < 1.05, fp32
     assert 0.60 < sfu / (sms * 16 * clk_hz) < 1.05, sfu
     assert B.lib.idkm_measure_pipe_rates(None, None, None) == B.ERR_NULL
+
+
+@pytest.mark.parametrize("d,k,m", [(1, 4, 4096), (1, 8, 36864), (2, 2, 50001), (4, 8, 100000), (1, 4, 1 << 20)])
+def test_one_launch_forward_loop_matches_launch_per_iteration(d, k, m):
+    """The cooperative one-launch forward loop and the launch-per-iteration loop run the same iteration: both match
+    the oracle, they agree with each other far inside the tolerance, the one-launch path really is one launch, and a
+    tolerance-mode run stops at the same iteration count."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(m, d, k, 0.01, std=0.03, seed=11, max_iter=12)
+    dev = torch.device("cuda:0")
+    W, C0 = torch.from_numpy(wl.W).to(dev), torch.from_numpy(wl.C0).to(dev)
+    ref = oracle_run(wl, want_dW=False)
+    outs = {}
+    for method in (0, 1):
+        ctx = B.Context()
+        ctx.set_forward_loop(method)
+        n0 = ctx.launches
+        fr = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter, want_Wq=True)
+        torch.cuda.synchronize()
+        outs[method] = (fr.C.cpu().numpy().astype(np.float64), ctx.launches - n0, ctx.info()[0])
+        assert_close(outs[method][0], ref["C"], TOL_C, f"C, loop method {method}")
+        assert outs[method][2].fwd_iters == wl.max_iter and outs[method][2].status == 0
+    assert outs[0][1] == 3                       # init, the loop, the final pass
+    assert outs[1][1] == 2 + 2 * wl.max_iter     # init, (fp32 + fp64 step) per iteration, the final pass
+    assert_close(outs[0][0], outs[1][0], 1e-6, "one-launch vs per-iteration centroids")
+    # tolerance mode: same stopping iteration
+    its = []
+    for method in (0, 1):
+        ctx = B.Context()
+        ctx.set_forward_loop(method)
+        ctx.forward(W, C0, wl.tau, 1e-4, 200)
+        torch.cuda.synchronize()
+        its.append(ctx.info()[0].fwd_iters)
+    assert its[0] == its[1] and 1 <= its[0] <= 200
