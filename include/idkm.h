@@ -209,8 +209,9 @@ int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
 int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_per_s, void* cuda_stream);
 
 /*
- * How the forward loop (Algorithm 1) is launched.  0 (default): a single layer with k <= 8 and at most about 2.4
- * million rows (32 rows per thread of the co-resident grid) runs the WHOLE loop in one cooperative launch: per
+ * How the forward loop (Algorithm 1) is launched.  0 (default): a single layer with k <= 16 (k <= 8 for d = 4) and
+ * at most about 4.8 million rows (64 rows per thread of the co-resident grid) runs the WHOLE loop in one cooperative
+ * launch: per
  * iteration every block publishes one fp64 partial, all blocks meet at a grid-wide barrier, and every block then
  * adds the partials in the same order and takes the M-step itself, so only the partials cross L2 inside the loop;
  * the loop leaves at the iteration whose stop test passes.  Everything else (batched layers, larger layers or

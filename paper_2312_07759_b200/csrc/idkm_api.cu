@@ -22,12 +22,15 @@ extern const KernelEntry k_table_scatter[3][N_FAMILY];
 extern const KernelEntry k_table_step_precise[3][N_FAMILY];
 extern const KernelEntry k_table_jacobian[3][N_FAMILY];
 extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY];
+extern const DualEntry k_table_dual[3][2];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
-                                  double inv_tau, unsigned int* gtickets, int n_groups, unsigned int* sync) {
+                                  double inv_tau, unsigned int* gtickets, int n_groups, unsigned int* sync,
+                                  unsigned int* gtickets64, int n_groups64) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   for (int o = i; o < n_groups; o += gridDim.x * blockDim.x) gtickets[o] = 0u;
+  for (int o = i; o < n_groups64; o += gridDim.x * blockDim.x) gtickets64[o] = 0u;
   if (i < 4) sync[i] = 0u;
   if (i < n_layers) {
     LayerState s;
@@ -107,9 +110,20 @@ int pick_family(int mode, int d, int k) {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The dual step kernel of (d, k), or null: it exists for the layouts (2,1) and (4,1) where the fp32 and the fp64 step
+// pick the same layout and register budget.
+static const DualEntry* dual_entry(int d, int k) {
+  const int di = d == 1 ? 0 : (d == 2 ? 1 : (d == 4 ? 2 : -1));
+  const int f = pick_family(STEP, d, k);
+  if (di < 0 || f < 0 || f > 1 || pick_family(STEP_PRECISE, d, k) != f) return nullptr;
+  const DualEntry* e = &k_table_dual[di][f];
+  return e->launch ? e : nullptr;
+}
+
 struct WorkspaceLayout {
   size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, off_sync, total;
-  int max_slots, max_groups;
+  size_t off_partials64, off_gpartials64, off_gtickets64;   // second set for the fp64 half of the dual step kernel
+  int max_slots, max_groups, max_groups64;
 };
 
 static int device_sm_count() {
@@ -145,6 +159,12 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   w.off_gpartials = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups * plen_max, 256);
   w.off_gtickets = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups, 256);
   w.off_sync = o;      o = align_up(o + 4 * sizeof(unsigned int), 256);   // barrier words of the single-launch loop
+  const DualEntry* de = dual_entry(d, k);
+  const int plen64 = de ? kernel_entry(STEP_PRECISE, d, pick_family(STEP_PRECISE, d, k))->plen : 0;
+  w.max_groups64 = de ? w.max_groups : 0;
+  w.off_partials64 = o;  o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen64, 256);
+  w.off_gpartials64 = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups64 * plen64, 256);
+  w.off_gtickets64 = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups64, 256);
   w.total = o;
   *out = w;
   return true;
@@ -296,35 +316,55 @@ struct RunAhead {
 
 // The forward loop: every iteration launches the fp32 step and the fp64 step; each layer is taken by exactly one
 // of them (LayerState::precise), the other returns at once for it.
-static int launch_step_loop(idkm_ctx* ctx, PassParams* p, int repeat) {
+static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p, int repeat) {
   const int f32 = pick_family(STEP, ctx->d, ctx->k), f64 = pick_family(STEP_PRECISE, ctx->d, ctx->k);
   const KernelEntry* e32 = kernel_entry(STEP, ctx->d, f32);
   const KernelEntry* e64 = kernel_entry(STEP_PRECISE, ctx->d, f64);
+  static const bool dual_off = (getenv("IDKM_NO_DUAL") != nullptr);   // tuning knob: always two launches per iteration
+  const DualEntry* de = dual_off ? nullptr : dual_entry(ctx->d, ctx->k);
   PassParams q = *p;
   int rc = build_table(ctx, STEP, f32, &p->lt);
   if (rc != IDKM_OK) return rc;
   rc = build_table(ctx, STEP_PRECISE, f64, &q.lt);
   if (rc != IDKM_OK) return rc;
+  int dual_grid = 0;
+  if (de) {
+    // one grid runs both halves: each half's table may use at most that many blocks
+    char* ws = static_cast<char*>(ctx->workspace);
+    q.partials = reinterpret_cast<double*>(ws + wl.off_partials64);
+    q.gpartials = reinterpret_cast<double*>(ws + wl.off_gpartials64);
+    q.gtickets = reinterpret_cast<unsigned int*>(ws + wl.off_gtickets64);
+    dual_grid = p->lt.n_blocks > q.lt.n_blocks ? p->lt.n_blocks : q.lt.n_blocks;
+  }
   RunAhead ra;
   ra.begin(ctx, p, p->tol > 0.f);
   q.host_flag = p->host_flag;
   q.call_id = p->call_id;
   for (int it = 0; it < repeat; ++it) {
     p->iter = q.iter = it;
-    if (e32->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
-    if (e64->launch(q, q.lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
-    ctx->launches += 2;
+    if (de) {
+      DualParams dp;
+      dp.p = *p;
+      dp.q = q;
+      if (de->launch(dp, dual_grid, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+      ctx->launches += 1;
+    } else {
+      if (e32->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+      if (e64->launch(q, q.lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+      ctx->launches += 2;
+    }
     if (ra.after(it)) break;
   }
   p->host_flag = nullptr;
   return IDKM_OK;
 }
 
-// The single-launch loop takes a single layer with k <= 8 whose rows fit SMALL_ROWS_PER_THREAD per thread of the
-// co-resident grid (so that a thread's fp32 sums stay short, as in the tiled passes) -- about 2.4 million rows on a
-// 148-SM part.  Blocks get at least SMALL_MIN_ROWS_PER_THREAD rows per thread: tiny layers use few blocks, which keeps
+// The single-launch loop takes a single layer with k <= 16 (k <= 8 for d = 4) whose rows fit SMALL_ROWS_PER_THREAD per
+// thread of the co-resident grid -- about 4.8 million rows on a 148-SM part (beyond that the tiled step kernels with
+// their deeper load pipelines are faster).  Blocks get at least SMALL_MIN_ROWS_PER_THREAD rows per thread: tiny layers use few blocks, which keeps
 // the cross-block sum short.
-constexpr int SMALL_ROWS_PER_THREAD = 32;
+constexpr int SMALL_ROWS_PER_THREAD = 64;
+constexpr int SMALL_CHUNK_ROWS = 32;   // threads with more rows than this move their fp32 sums out every 32 rows
 constexpr int SMALL_MIN_ROWS_PER_THREAD = 4;
 constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM clock ticks per barrier wait
 
@@ -335,7 +375,7 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   const int di = d_index(ctx->d);
   int f = -1;
   for (int q = 0; q < N_SMALL_FAMILY; ++q)
-    if (k_table_small[di][q].kpl >= ctx->k) { f = q; break; }
+    if (k_table_small[di][q].launch && k_table_small[di][q].kpl >= ctx->k) { f = q; break; }
   if (f < 0) return 1;
   const SmallLoopEntry* se = &k_table_small[di][f];
   int& nb = ctx->small_blocks[di][f];
@@ -343,7 +383,8 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
     int coop = 0, per_sm = 0;
     nb = -1;
     if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, se->func, BLOCK, 0) == cudaSuccess && per_sm >= 1)
+        cudaFuncSetAttribute(se->func, cudaFuncAttributeMaxDynamicSharedMemorySize, se->dyn_smem) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, se->func, BLOCK, se->dyn_smem) == cudaSuccess && per_sm >= 1)
       nb = ctx->sms * (per_sm > 2 ? 2 : per_sm);
     (void)cudaGetLastError();
   }
@@ -367,6 +408,7 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   sp.tol = p.tol;
   sp.inv_tau_d = p.inv_tau_d;
   sp.max_iter = max_iter;
+  sp.chunked = (m > (long long)SMALL_CHUNK_ROWS * grid * BLOCK) ? 1 : 0;
   sp.spin_limit = SMALL_SPIN_LIMIT;
   if (se->launch(sp, (int)grid, ctx->stream) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -486,13 +528,15 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
   const int init_threads = n_coord > n_layers ? n_coord : n_layers;
   idkm_init_forward<<<(init_threads + 255) / 256, 256, 0, ctx->stream>>>(p.st, n_layers, C0, C_out, n_coord, k, d,
                                                                                      p.inv_tau_d, p.gtickets, wl.max_groups,
-                                                                                     reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + wl.off_sync));
+                                                                                     reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + wl.off_sync),
+                                                                                     reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + wl.off_gtickets64),
+                                                                                     wl.max_groups64);
   if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
   ++ctx->launches;
   mark(ctx, 1);
 
   int rc = try_small_loop(ctx, wl, p, max_iter);
-  if (rc == 1) rc = launch_step_loop(ctx, &p, max_iter);
+  if (rc == 1) rc = launch_step_loop(ctx, wl, &p, max_iter);
   if (rc != IDKM_OK) return rc;
   mark(ctx, 2);
   p.Wq = Wq_out;

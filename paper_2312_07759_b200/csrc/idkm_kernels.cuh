@@ -475,9 +475,11 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
 }
 
 // ---- the pass ------------------------------------------------------------------------------------
-template <int MODE, int D, int KPL, int LPW>
-__global__ void __launch_bounds__(BLOCK, PassCfg<MODE, D, KPL, LPW>::MIN_BLOCKS)
-idkm_pass(const __grid_constant__ PassParams p) {
+// RELEASE: let the next kernel of the stream be scheduled once this block's rows are done (the caller has already
+// waited for the previous kernel).  The dual step kernel runs this body with RELEASE = false and releases after its
+// second body.
+template <int MODE, int D, int KPL, int LPW, bool RELEASE>
+__device__ __forceinline__ void pass_body(const PassParams& p) {
   using Cfg = PassCfg<MODE, D, KPL, LPW>;
   constexpr int NACC = Cfg::NACC;
   constexpr int PLEN = Cfg::PLEN;
@@ -508,7 +510,6 @@ idkm_pass(const __grid_constant__ PassParams p) {
   __shared__ __align__(16) float gstage[NEED_G ? STAGE : 4];
   (void)wstage; (void)gstage;
 
-  grid_dependency_sync();
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
@@ -519,7 +520,7 @@ idkm_pass(const __grid_constant__ PassParams p) {
   const int b = blockIdx.x;
   const int t_lo = tile_begin(b, p.lt.tiles_total, nb);
   const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
-  if (t_lo >= t_hi) return;
+  if (b >= nb || t_lo >= t_hi) return;   // (the dual step kernel's grid can be larger than this pass's table)
 
   // Centroids and sums are held as float2 pairs of neighbouring centroids (2h, 2h+1); c_(t, a) / acc_(t, a) give
   // the scalar view, which resolves to a register half once the loops are unrolled.  (The packed fp32x2
@@ -964,8 +965,15 @@ idkm_pass(const __grid_constant__ PassParams p) {
       }
     }
   }
-  grid_release_dependents();
+  if constexpr (RELEASE) grid_release_dependents();
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
+}
+
+template <int MODE, int D, int KPL, int LPW>
+__global__ void __launch_bounds__(BLOCK, PassCfg<MODE, D, KPL, LPW>::MIN_BLOCKS)
+idkm_pass(const __grid_constant__ PassParams p) {
+  grid_dependency_sync();
+  pass_body<MODE, D, KPL, LPW, true>(p);
 }
 
 
@@ -1014,8 +1022,7 @@ __device__ __forceinline__ double group_sum_d(double v) {
 }
 
 template <int D, int KPL, int LPW>
-__global__ void __launch_bounds__(BLOCK, PreciseCfg<D, KPL, LPW>::MIN_BLOCKS)
-idkm_step_precise(const __grid_constant__ PassParams p) {
+__device__ __forceinline__ void precise_body(const PassParams& p) {
   using Cfg = PreciseCfg<D, KPL, LPW>;
   constexpr int NA = Cfg::NA;
   constexpr int PLEN = Cfg::PLEN;
@@ -1027,7 +1034,6 @@ idkm_step_precise(const __grid_constant__ PassParams p) {
   __shared__ __align__(16) unsigned char smem_raw[SMEM_BYTES];
   __shared__ int s_flag;
 
-  grid_dependency_sync();
   const int tid = threadIdx.x;
   const int lane = tid & 31;
   const int warp = tid >> 5;
@@ -1038,7 +1044,7 @@ idkm_step_precise(const __grid_constant__ PassParams p) {
   const int b = blockIdx.x;
   const int t_lo = tile_begin(b, p.lt.tiles_total, nb);
   const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
-  if (t_lo >= t_hi) return;
+  if (b >= nb || t_lo >= t_hi) return;   // (the dual step kernel's grid can be larger than this pass's table)
 
   double c[KPL][D];
   double acc[KPL][NA];
@@ -1177,6 +1183,31 @@ idkm_step_precise(const __grid_constant__ PassParams p) {
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
 }
 
+template <int D, int KPL, int LPW>
+__global__ void __launch_bounds__(BLOCK, PreciseCfg<D, KPL, LPW>::MIN_BLOCKS)
+idkm_step_precise(const __grid_constant__ PassParams p) {
+  grid_dependency_sync();
+  precise_body<D, KPL, LPW>(p);
+}
+
+// One launch per forward iteration instead of two, for the smallest thread-per-weight layouts, where the fp32 and
+// the fp64 step have the same register budget: every block first takes its tiles of the layers that step in fp32,
+// then its tiles of the layers that step in fp64 (own tile table, own partial-sum buffers: the two run side by side
+// across blocks).  On a batched workload with collapsing layers the two kinds of layers then overlap instead of
+// running one kernel after the other.
+struct DualParams {
+  PassParams p;   // fp32 step
+  PassParams q;   // fp64 step
+};
+template <int D, int KPL>
+__global__ void __launch_bounds__(BLOCK, PreciseCfg<D, KPL, 1>::MIN_BLOCKS)
+idkm_step_dual(const __grid_constant__ DualParams dp) {
+  grid_dependency_sync();
+  pass_body<STEP, D, KPL, 1, false>(dp.p);
+  __syncthreads();
+  precise_body<D, KPL, 1>(dp.q);
+}
+
 
 // ---- explicit Jacobian for small codebooks -------------------------------------------------------------------
 // When k d <= 8 the matrix J_C = dF/dC (k d x k d, at most 64 entries) fits in a thread's registers.  One pass over
@@ -1212,7 +1243,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_jacobian(const __grid_constant__ P
   const int b = blockIdx.x;
   const int t_lo = tile_begin(b, p.lt.tiles_total, nb);
   const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
-  if (t_lo >= t_hi) return;
+  if (b >= nb || t_lo >= t_hi) return;   // (the dual step kernel's grid can be larger than this pass's table)
 
   float c[KPL][D], fj[KPL][D], ist[KPL];   // centroids, F(C_T, W)_j, 1 / (S_j tau) (0 for a dead or padding cluster)
   float jac[KD][KD];
@@ -1447,7 +1478,14 @@ struct KernelEntry {
   int kpl, lpw, tile, plen;
   int dyn_smem;   // dynamic shared memory the launch asks for (bytes)
 };
-// Single-launch forward loop for one small layer (idkm_small_loop.cu): k <= 2, 4, 8 centroids per thread.
+// dual step kernel (idkm_pass_step_dual.cu): exists where PreciseCfg<D, KPL, 1>::MIN_BLOCKS == 4
+typedef cudaError_t (*DualLaunchFn)(const DualParams& dp, int grid, cudaStream_t stream);
+struct DualEntry {
+  DualLaunchFn launch;
+  const void* func;
+  int dyn_smem;
+};
+// Single-launch forward loop for one small layer (idkm_small_loop.cu): k <= 2, 4, 8, 16 centroids per thread.
 struct SmallLoopParams {
   const float* W;
   long long m;
@@ -1460,15 +1498,16 @@ struct SmallLoopParams {
   float tol;
   double inv_tau_d;
   int max_iter;
+  int chunked;           // 1: some thread has more than 32 rows, fp32 sums are moved out every 32 rows
   long long spin_limit;  // clock64() ticks a block waits at a barrier before it gives up
 };
 typedef cudaError_t (*SmallLaunchFn)(const SmallLoopParams& sp, int grid, cudaStream_t stream);
 struct SmallLoopEntry {
   SmallLaunchFn launch;
   const void* func;
-  int kpl, plen;
+  int kpl, plen, dyn_smem;
 };
-constexpr int N_SMALL_FAMILY = 3;
+constexpr int N_SMALL_FAMILY = 4;
 // family index f: 0..7 -> supports k <= kpl*lpw
 constexpr int N_FAMILY = 9;
 const KernelEntry* kernel_entry(int mode, int d, int family);

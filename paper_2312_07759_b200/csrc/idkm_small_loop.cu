@@ -1,4 +1,4 @@
-// Algorithm 1's whole loop in ONE cooperative launch, for a single small layer (k <= 8, a few million weights at most).
+// Algorithm 1's whole loop in ONE cooperative launch, for a single small layer (k <= 16, a few million weights at most).
 //
 // There one iteration is a few microseconds of arithmetic, and a launch per iteration -- with its chain of dependent
 // trips to L2 (partials, ticket, totals, centroids, state) -- costs more than the arithmetic.  Here all blocks are
@@ -11,12 +11,15 @@
 
 namespace idkm {
 
+constexpr int SMALL_CHUNK = 32;   // rows a thread adds into one fp32 accumulator before it moves the sum out
+
 template <int D, int KPL>
 struct SmallCfg {
   static constexpr int NA = D + 1;
   static constexpr int PLEN = KPL * NA;
   static constexpr int CH = BLOCK / PLEN;          // chunks of partial rows added in parallel in the second level
   static constexpr int KD = KPL * D;
+  static constexpr int DYN_SMEM = PLEN * BLOCK * 4;
 };
 
 // Bounded wait until the arrival counter has reached `target`.  Returns false if the wait ran out or another block
@@ -44,7 +47,8 @@ __device__ __forceinline__ bool small_barrier(unsigned int* sync, unsigned int t
   return *s_ok != 0;
 }
 
-template <int D, int KPL>
+// CHUNKED: some thread has more than SMALL_CHUNK rows; its fp32 sums are then moved out every SMALL_CHUNK rows.
+template <int D, int KPL, bool CHUNKED>
 __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constant__ SmallLoopParams sp) {
   using Cfg = SmallCfg<D, KPL>;
   constexpr int NA = Cfg::NA, PLEN = Cfg::PLEN, CH = Cfg::CH, KD = Cfg::KD;
@@ -55,6 +59,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
   __shared__ float c_sm[KD > 0 ? KD : 1];   // the current centroids (every block holds the same values)
   __shared__ double s_res[4];       // residual, dead, bad, box2
   __shared__ int s_ok;
+  extern __shared__ __align__(16) float slots[];   // [PLEN][BLOCK] second-level fp32 sums (CHUNKED only)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int b = blockIdx.x, G = gridDim.x;
@@ -96,10 +101,37 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
 #pragma unroll
       for (int t = 0; t < KPL; ++t)
 #pragma unroll
-        for (int a = 0; a < NA; ++a) acc[t][a] = 0.f;
-      for (long long r = (long long)b * BLOCK + tid; r < m; r += (long long)G * BLOCK) {
+        for (int a = 0; a < NA; ++a) {
+          acc[t][a] = 0.f;
+          if constexpr (CHUNKED) slots[(t * NA + a) * BLOCK + tid] = 0.f;
+        }
+      int since = 0;
+      const long long stride = (long long)G * BLOCK;
+      const long long r_first = (long long)b * BLOCK + tid;
+      float wn[D];   // the next row, fetched while the current one is processed
+#pragma unroll
+      for (int a = 0; a < D; ++a) wn[a] = 0.f;
+      if (r_first < m) load_row(r_first, wn);
+      for (long long r = r_first; r < m; r += stride) {
+        // A long fp32 running sum drops the many terms below half its ulp (one-sided): threads with more than
+        // SMALL_CHUNK rows move their sums into a private shared-memory slot every SMALL_CHUNK rows.
+        if constexpr (CHUNKED) {
+          if (since == SMALL_CHUNK) {
+#pragma unroll
+            for (int t = 0; t < KPL; ++t)
+#pragma unroll
+              for (int a = 0; a < NA; ++a) {
+                slots[(t * NA + a) * BLOCK + tid] += acc[t][a];
+                acc[t][a] = 0.f;
+              }
+            since = 0;
+          }
+          ++since;
+        }
         float w[D];
-        load_row(r, w);
+#pragma unroll
+        for (int a = 0; a < D; ++a) w[a] = wn[a];
+        if (r + stride < m) load_row(r + stride, wn);
         float dist[KPL], e[KPL];
 #pragma unroll
         for (int t = 0; t < KPL; ++t) {
@@ -134,6 +166,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
 #pragma unroll
         for (int a = 0; a < NA; ++a) {
           float v = acc[t][a];
+          if constexpr (CHUNKED) v += slots[(t * NA + a) * BLOCK + tid];
 #pragma unroll
           for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
           if (lane == 0) red[warp][t * NA + a] = v;
@@ -305,13 +338,28 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
 
 template <int D, int KPL>
 static cudaError_t launch_small(const SmallLoopParams& sp, int grid, cudaStream_t stream) {
+  constexpr int DYN = SmallCfg<D, KPL>::DYN_SMEM;
+  static bool configured = false;   // the slots of the widest layouts reach the 48 KB default limit
+  if (!configured) {
+    const cudaError_t rc = cudaFuncSetAttribute(idkm_small_loop<D, KPL, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DYN);
+    if (rc != cudaSuccess) return rc;
+    configured = true;
+  }
   void* args[1] = {const_cast<SmallLoopParams*>(&sp)};
   // cooperative launch: refused (instead of hanging at the first barrier) if the grid cannot be co-resident
-  return cudaLaunchCooperativeKernel((const void*)&idkm_small_loop<D, KPL>, dim3((unsigned)grid, 1, 1),
+  if (sp.chunked)
+    return cudaLaunchCooperativeKernel((const void*)&idkm_small_loop<D, KPL, true>, dim3((unsigned)grid, 1, 1),
+                                       dim3(BLOCK, 1, 1), args, (size_t)DYN, stream);
+  return cudaLaunchCooperativeKernel((const void*)&idkm_small_loop<D, KPL, false>, dim3((unsigned)grid, 1, 1),
                                      dim3(BLOCK, 1, 1), args, 0, stream);
 }
-#define IDKM_SMALL_ENTRY(D, KPL) { &launch_small<D, KPL>, (const void*)&idkm_small_loop<D, KPL>, KPL, SmallCfg<D, KPL>::PLEN }
-#define IDKM_SMALL_ROW(D) { IDKM_SMALL_ENTRY(D, 2), IDKM_SMALL_ENTRY(D, 4), IDKM_SMALL_ENTRY(D, 8) }
-extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY] = {IDKM_SMALL_ROW(1), IDKM_SMALL_ROW(2), IDKM_SMALL_ROW(4)};
+#define IDKM_SMALL_ENTRY(D, KPL) \
+  { &launch_small<D, KPL>, (const void*)&idkm_small_loop<D, KPL, true>, KPL, SmallCfg<D, KPL>::PLEN, SmallCfg<D, KPL>::DYN_SMEM }
+#define IDKM_SMALL_NONE { nullptr, nullptr, 0, 0, 0 }
+// 16 centroids per thread only for d = 1, 2: with d = 4 the centroids and sums alone exceed the register budget
+extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY] = {
+    {IDKM_SMALL_ENTRY(1, 2), IDKM_SMALL_ENTRY(1, 4), IDKM_SMALL_ENTRY(1, 8), IDKM_SMALL_ENTRY(1, 16)},
+    {IDKM_SMALL_ENTRY(2, 2), IDKM_SMALL_ENTRY(2, 4), IDKM_SMALL_ENTRY(2, 8), IDKM_SMALL_ENTRY(2, 16)},
+    {IDKM_SMALL_ENTRY(4, 2), IDKM_SMALL_ENTRY(4, 4), IDKM_SMALL_ENTRY(4, 8), IDKM_SMALL_NONE}};
 
 }  // namespace idkm
