@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "libidkm.so")
 
-HEADERS = ["idkm_kernels.cuh", "idkm_inst.cuh", os.path.join(ROOT, "include", "idkm.h")]
+HEADERS = ["idkm_kernels.cuh", "idkm_inst.cuh", "idkm_jacobian_tile.cuh", os.path.join(ROOT, "include", "idkm.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
               "-diag-suppress", "177"]

@@ -110,6 +110,13 @@ int pick_family(int mode, int d, int k) {
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// The explicit-Jacobian pass comes in two kinds: k d <= 8 (matrix in a thread's registers, at most 64 entries) and
+// the tiled kind for k d <= 64, whose partials are whole matrices and which therefore runs two blocks per SM.
+constexpr int JAC_SMALL_PLEN_MAX = 64;
+constexpr int JAC_TILE_BLOCKS_PER_SM = 2;
+// Steps of the adjoint iteration from which the tiled kind (one pass of about ten fused passes' cost) is used.
+constexpr int JAC_TILE_MIN_ITERS = 16;
+
 // The dual step kernel of (d, k), or null: it exists for the layouts (2,1) and (4,1) where the fp32 and the fp64 step
 // pick the same layout and register budget.
 static const DualEntry* dual_entry(int d, int k) {
@@ -139,11 +146,16 @@ static int device_sm_count() {
 static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* out) {
   if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K || n_layers < 1 || n_layers > IDKM_MAX_LAYERS) return false;
   int plen_max = 1;
+  size_t jac_tile_doubles = 0;   // the tiled explicit-Jacobian pass: k d x k d partials, but only two blocks per SM
   for (int mode = STEP; mode < N_MODES; ++mode) {
     const int f = pick_family(mode, d, k);
     if (f < 0 && mode == JACOBIAN) continue;   // only small codebooks have the explicit-Jacobian pass
     if (f < 0) return false;
     const int pl = kernel_entry(mode, d, f)->plen;
+    if (mode == JACOBIAN && pl > JAC_SMALL_PLEN_MAX) {
+      jac_tile_doubles = (size_t)(sms * JAC_TILE_BLOCKS_PER_SM + n_layers) * pl;
+      continue;
+    }
     if (pl > plen_max) plen_max = pl;
   }
   WorkspaceLayout w;
@@ -154,7 +166,9 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   w.off_g = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k * d, 256);
   w.off_u = o;     o = align_up(o + sizeof(float) * (size_t)n_layers * k * d, 256);
   w.max_slots = sms * MAX_BLOCKS_PER_SM + n_layers;
-  w.off_partials = o; o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen_max, 256);
+  size_t partial_doubles = (size_t)w.max_slots * plen_max;
+  if (jac_tile_doubles > partial_doubles) partial_doubles = jac_tile_doubles;
+  w.off_partials = o; o = align_up(o + sizeof(double) * partial_doubles, 256);
   w.max_groups = w.max_slots / RED_GROUP + n_layers + 2;
   w.off_gpartials = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups * plen_max, 256);
   w.off_gtickets = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups, 256);
@@ -250,6 +264,8 @@ static int build_table(idkm_ctx* ctx, int mode, int family, LayerTable* lt) {
   }
   lt->tiles_total = (int)tiles;
   long long nb = (long long)ctx->sms * blocks_per_sm(ctx, mode, ctx->d, family);
+  if (mode == JACOBIAN && e->plen > JAC_SMALL_PLEN_MAX && nb > (long long)ctx->sms * JAC_TILE_BLOCKS_PER_SM)
+    nb = (long long)ctx->sms * JAC_TILE_BLOCKS_PER_SM;   // the workspace holds this many matrix partials
   // Batched loops: layers drop out of a loop at different times (converged, or handed to the other step kernel),
   // and the blocks that own their tiles return at once.  With more blocks than fit on the GPU at a time the
   // hardware scheduler backfills the freed slots with blocks of the layers that still run, instead of leaving SMs
@@ -585,7 +601,9 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   if (rc != IDKM_OK) return rc;
   mark(ctx, 5);
   if (mode == IDKM_IMPLICIT && adj_max_iter > 0) {
-    if (ctx->adjoint_method == 0 && pick_family(JACOBIAN, ctx->d, ctx->k) >= 0)
+    const int fj = pick_family(JACOBIAN, ctx->d, ctx->k);
+    const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, ctx->d, fj)->plen > JAC_SMALL_PLEN_MAX;
+    if (ctx->adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS))
       rc = launch_pass(ctx, JACOBIAN, &p, 1);      // one pass forms J_C; the whole iteration runs on it in the epilogue
     else
       rc = launch_pass(ctx, ADJ, &p, adj_max_iter);

@@ -90,13 +90,18 @@ def test_non_default_stream():
     assert_close(dW.cpu().numpy(), ref["dW"], TOL_GRAD, "dW")
 
 
-@pytest.mark.parametrize("m,d,k", [(30001, 1, 4), (20000, 1, 8), (10000, 2, 4), (9000, 4, 2), (5000, 2, 3)])
+@pytest.mark.parametrize("m,d,k", [(30001, 1, 4), (20000, 1, 8), (10000, 2, 4), (9000, 4, 2), (5000, 2, 3),
+                                   (40000, 1, 16), (33333, 2, 16), (50000, 4, 16), (20001, 1, 64), (25000, 2, 32),
+                                   (12345, 4, 5), (300000, 1, 12), (7000, 2, 7), (31, 4, 3)])
 def test_explicit_jacobian_adjoint_equals_fused_passes(m, d, k):
-    """For k*d <= 8 the adjoint iteration runs on the explicitly formed k d x k d matrix (one pass over W); it must
-    give the iterates of the one-pass-per-step path, with the tolerance rule and the counters behaving the same."""
+    """For k*d <= 64 the adjoint iteration runs on the explicitly formed k d x k d matrix (one pass over W; for
+    k*d > 8 from 16 steps on); it must give the iterates of the one-pass-per-step path, with the tolerance rule and
+    the counters behaving the same."""
     import torch
     from paper_2312_07759_b200 import binding as B
-    wl = WL.single_layer(m, d, k, 0.012, std=0.03, seed=m + k, max_iter=15, adj_max_iter=12, init="rows", g_std=0.3)
+    adj_iters = 12 if k * d <= 8 else 20
+    wl = WL.single_layer(m, d, k, 0.012, std=0.03, seed=m + k, max_iter=15, adj_max_iter=adj_iters, init="rows",
+                         g_std=0.3)
     W, C0, G = (torch.from_numpy(x).cuda() for x in (wl.W, wl.C0, wl.G))
     res = {}
     for method in (0, 1):
