@@ -190,10 +190,12 @@ int idkm_step_noalloc(const float* W, int64_t m, int d, const float* C_in, int k
                       void* cuda_stream);
 
 /*
- * How IDKM_IMPLICIT runs the adjoint iteration.  0 (default): where k d <= 8 one pass over W forms the k d x k d
+ * How IDKM_IMPLICIT runs the adjoint iteration.  0 (default): where k d <= 64 one pass over W forms the k d x k d
  * matrix dF/dC explicitly and the whole iteration u <- alpha (J^T u + g) + (1 - alpha) u then runs on that matrix on
  * the device -- the paper's own formulation (it iterates a k x k matrix, Section 4.2), same iterates, one pass
- * instead of adj_max_iter; larger codebooks use one fused vector-Jacobian pass per step.  1: always the fused passes.
+ * instead of adj_max_iter.  For k d <= 8 always; for 8 < k d <= 64 (the pass costs about ten fused passes) when
+ * adj_max_iter >= 16.  Larger codebooks, and shorter iterations, use one fused vector-Jacobian pass per step.
+ * 1: always the fused passes.
  */
 int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
 
