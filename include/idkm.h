@@ -200,6 +200,22 @@ int idkm_step_noalloc(const float* W, int64_t m, int d, const float* C_in, int k
 int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
 
 /*
+ * Hard assignment, q(w) = argmin_c ||w - c|| (Section 3.1: the map the soft quantiser r_tau of the forward tends
+ * to as tau -> 0) -- the codes and dequantised weights of the trained layer.  For every row i of W [m][d] (DEVICE,
+ * fp32) the index of the nearest row of C [k][d] (DEVICE, fp32; squared distances in fp32, ties to the lowest index)
+ * is written to codes_out (DEVICE, idkm_codes_bytes(m, k) bytes, or NULL): b = idkm_code_bits(k) bits per weight,
+ * b the smallest of 1, 2, 4, 8 with 2^b >= k, at bit offset (i b) mod 8 of byte (i b) / 8 (little-endian within the
+ * byte; unused high bits of the last byte are 0).  Wq_out (DEVICE [m][d], or NULL; not W) receives the assigned
+ * centroid of every row.  At least one output must be given.  d in {1,2,4}, 1 <= k <= 256, m >= 1; needs no
+ * context and no workspace and allocates nothing; asynchronous on cuda_stream.
+ * Returns IDKM_OK, IDKM_ERR_NULL, IDKM_ERR_UNSUPPORTED, IDKM_ERR_SHAPE, IDKM_ERR_PARAM or IDKM_ERR_CUDA.
+ */
+int idkm_assign(const float* W, int64_t m, int d, const float* C, int k, unsigned char* codes_out, float* Wq_out,
+                void* cuda_stream);
+int idkm_code_bits(int k);                   /* 1, 2, 4 or 8; 0 for k outside [1, 256] */
+size_t idkm_codes_bytes(int64_t m, int k);   /* ceil(m * idkm_code_bits(k) / 8); 0 for bad arguments */
+
+/*
  * Measured issue rates of the two pipes that bound the arithmetic-bound passes, for roofline denominators (the
  * paper has no counterpart: this is a measurement utility, nothing on the IDKM path calls it).  Two register-only
  * kernels over all SMs -- eight independent chains per thread of fp32 fused multiply-adds, and of ex2.approx --

@@ -68,6 +68,12 @@ lib.idkm_launch_count.argtypes = [_vp]
 lib.idkm_launch_count.restype = C.c_int64
 lib.idkm_measure_pipe_rates.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), _vp]
 lib.idkm_measure_pipe_rates.restype = C.c_int
+lib.idkm_assign.argtypes = [_fp, C.c_int64, C.c_int, _fp, C.c_int, _vp, _fp, _vp]
+lib.idkm_assign.restype = C.c_int
+lib.idkm_code_bits.argtypes = [C.c_int]
+lib.idkm_code_bits.restype = C.c_int
+lib.idkm_codes_bytes.argtypes = [C.c_int64, C.c_int]
+lib.idkm_codes_bytes.restype = C.c_size_t
 lib.idkm_status_string.argtypes = [C.c_int]
 lib.idkm_status_string.restype = C.c_char_p
 
@@ -120,6 +126,19 @@ def step_noalloc(W, C_in, tau: float, C_out=None, stream=None):
     _check(lib.idkm_step_noalloc(_ptr(W), int(W.shape[0]), int(W.shape[1]), _ptr(C_in), int(C_in.shape[0]),
                                  float(tau), _ptr(C_out), _stream(stream)))
     return C_out
+
+
+def assign(W, Cm, want_codes: bool = True, want_Wq: bool = True, stream=None):
+    """``idkm_assign``: packed nearest-centroid codes (uint8 CUDA tensor) and dequantised weights of CUDA fp32 W."""
+    import torch
+    assert W.is_cuda and Cm.is_cuda and W.dtype == torch.float32 and Cm.dtype == torch.float32
+    assert W.is_contiguous() and Cm.is_contiguous() and W.shape[1] == Cm.shape[1]
+    m, d, k = int(W.shape[0]), int(W.shape[1]), int(Cm.shape[0])
+    codes = torch.empty(int(lib.idkm_codes_bytes(m, k)), dtype=torch.uint8, device=W.device) if want_codes else None
+    Wq = torch.empty_like(W) if want_Wq else None
+    _check(lib.idkm_assign(_ptr(W), m, d, _ptr(Cm), k, _ptr(codes) if codes is not None else None,
+                           _ptr(Wq) if Wq is not None else None, _stream(stream)))
+    return codes, Wq
 
 
 def measure_pipe_rates(stream=None):
