@@ -206,9 +206,11 @@ int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
  * is written to codes_out (DEVICE, idkm_codes_bytes(m, k) bytes, or NULL): b = idkm_code_bits(k) bits per weight,
  * b the smallest of 1, 2, 4, 8 with 2^b >= k, at bit offset (i b) mod 8 of byte (i b) / 8 (little-endian within the
  * byte; unused high bits of the last byte are 0).  Wq_out (DEVICE [m][d], or NULL; not W) receives the assigned
- * centroid of every row.  At least one output must be given.  d in {1,2,4}, 1 <= k <= 256, m >= 1; needs no
+ * centroid of every row.  At least one output must be given; W and Wq_out 16-byte aligned.  d in {1,2,4},
+ * 1 <= k <= 256, m >= 1; needs no
  * context and no workspace and allocates nothing; asynchronous on cuda_stream.
- * Returns IDKM_OK, IDKM_ERR_NULL, IDKM_ERR_UNSUPPORTED, IDKM_ERR_SHAPE, IDKM_ERR_PARAM or IDKM_ERR_CUDA.
+ * Returns IDKM_OK, IDKM_ERR_NULL, IDKM_ERR_UNSUPPORTED, IDKM_ERR_SHAPE, IDKM_ERR_PARAM, IDKM_ERR_ALIGN or
+ * IDKM_ERR_CUDA.
  */
 int idkm_assign(const float* W, int64_t m, int d, const float* C, int k, unsigned char* codes_out, float* Wq_out,
                 void* cuda_stream);
