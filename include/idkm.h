@@ -238,6 +238,10 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
  * codebooks, max_iter < 2) takes one launch per iteration.  Every barrier wait is bounded (about a second): if one
  * runs out the kernel returns and the layer's status is IDKM_ERR_TIMEOUT.  1: always one launch per iteration.
  * Both run the same iteration; results differ only by the order of the cross-block sums.
+ *
+ * Test hooks for the timeout path (environment, read at every call; host-side fault injection only -- the waits stay
+ * bounded and the kernel returns): IDKM_TEST_MISSING_ARRIVALS=n makes each barrier wait for n arrivals that never
+ * come, IDKM_TEST_SPIN_LIMIT=ticks shortens the bound (SM clock ticks).
  */
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 

@@ -23,6 +23,7 @@ IMPLICIT, JFB = 0, 1
 OK, MAXITER = 0, 1
 ERR_NULL, ERR_ALIGN, ERR_SHAPE, ERR_UNSUPPORTED, ERR_PARAM = -1, -2, -3, -4, -5
 ERR_WORKSPACE, ERR_ORDER, ERR_CUDA, ERR_NONFINITE, ERR_DIVERGED = -6, -7, -8, -9, -10
+ERR_NOALLOC_TOO_LARGE, ERR_TIMEOUT = -11, -12
 
 
 class Info(C.Structure):

@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/idkm.h: argument checks, workspace layout, tile
 // tables and the launch sequences.  Every step of the path runs in the kernels of
 // idkm_kernels.cuh; nothing here computes on the data.
+#include <nvtx3/nvToolsExt.h>
 #include "idkm_kernels.cuh"
 
 #include <math.h>
@@ -426,6 +427,14 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   sp.max_iter = max_iter;
   sp.chunked = (m > (long long)SMALL_CHUNK_ROWS * grid * BLOCK) ? 1 : 0;
   sp.spin_limit = SMALL_SPIN_LIMIT;
+  // Host-side fault injection for tests of the timeout path (no GPU fault involved: the waits are bounded and the
+  // kernel returns): IDKM_TEST_MISSING_ARRIVALS=n makes every barrier wait for n arrivals that never come,
+  // IDKM_TEST_SPIN_LIMIT=ticks shortens the wait.  Both are read per call.
+  if (const char* e = getenv("IDKM_TEST_MISSING_ARRIVALS")) sp.missing_arrivals = atoi(e) > 0 ? atoi(e) : 0;
+  if (const char* e = getenv("IDKM_TEST_SPIN_LIMIT")) {
+    const long long v = atoll(e);
+    if (v > 0 && v < SMALL_SPIN_LIMIT) sp.spin_limit = v;
+  }
   if (se->launch(sp, (int)grid, ctx->stream) != cudaSuccess) {
     (void)cudaGetLastError();
     return 1;   // nothing was queued: take the launch-per-iteration path
@@ -551,13 +560,17 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
   ++ctx->launches;
   mark(ctx, 1);
 
+  nvtxRangePushA("idkm forward loop");
   int rc = try_small_loop(ctx, wl, p, max_iter);
   if (rc == 1) rc = launch_step_loop(ctx, wl, &p, max_iter);
+  nvtxRangePop();
   if (rc != IDKM_OK) return rc;
   mark(ctx, 2);
   p.Wq = Wq_out;
   p.A = A_out;
+  nvtxRangePushA("idkm final pass");
   rc = launch_pass(ctx, FINAL, &p, 1);
+  nvtxRangePop();
   if (rc != IDKM_OK) return rc;
   mark(ctx, 3);
   ctx->ev_fwd_set = ctx->timing && ctx->ev_ok;
@@ -597,22 +610,28 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   p.alpha = alpha;
   ctx->ev_bwd_set = false;
   mark(ctx, 4);
+  nvtxRangePushA("idkm codebook gradient");
   int rc = launch_pass(ctx, GRAD, &p, 1);
+  nvtxRangePop();
   if (rc != IDKM_OK) return rc;
   mark(ctx, 5);
   if (mode == IDKM_IMPLICIT && adj_max_iter > 0) {
     const int fj = pick_family(JACOBIAN, ctx->d, ctx->k);
     const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, ctx->d, fj)->plen > JAC_SMALL_PLEN_MAX;
+    nvtxRangePushA("idkm adjoint solve");
     if (ctx->adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS))
       rc = launch_pass(ctx, JACOBIAN, &p, 1);      // one pass forms J_C; the whole iteration runs on it in the epilogue
     else
       rc = launch_pass(ctx, ADJ, &p, adj_max_iter);
+    nvtxRangePop();
     if (rc != IDKM_OK) return rc;
   }
   mark(ctx, 6);
   if (dW_out) {
     p.dW = dW_out;
+    nvtxRangePushA("idkm dL/dW pass");
     rc = launch_pass(ctx, SCATTER, &p, 1);
+    nvtxRangePop();
     if (rc != IDKM_OK) return rc;
   }
   mark(ctx, 7);

@@ -1499,6 +1499,8 @@ struct SmallLoopParams {
   double inv_tau_d;
   int max_iter;
   int chunked;           // 1: some thread has more than 32 rows, fp32 sums are moved out every 32 rows
+  int missing_arrivals;  // 0 in production.  Host-side fault injection for the timeout path: the barriers wait for
+                         // this many arrivals more than the grid has, so every wait runs out (see idkm.h)
   long long spin_limit;  // clock64() ticks a block waits at a barrier before it gives up
 };
 typedef cudaError_t (*SmallLaunchFn)(const SmallLoopParams& sp, int grid, cudaStream_t stream);

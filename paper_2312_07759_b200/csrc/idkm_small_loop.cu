@@ -236,7 +236,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       }
     }
     // ---- everyone has published: grid-wide barrier ----
-    ok = small_barrier(sp.sync, (unsigned int)(it + 1) * (unsigned int)G, sp.spin_limit, &s_ok);
+    ok = small_barrier(sp.sync, (unsigned int)(it + 1) * (unsigned int)(G + sp.missing_arrivals), sp.spin_limit, &s_ok);
     if (!ok) break;
     // ---- every block adds all partials in the same order ----
     {
