@@ -138,6 +138,16 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
 int idkm_get_info(idkm_ctx* ctx, idkm_info* info_out);
 
 /*
+ * Residual history of the last forward (which = 0: relative change of C after each application of F, the quantity
+ * of the stop rule of Algorithm 1) or of the last implicit backward (which = 1: relative change of u after each
+ * adjoint step) of one layer.  Waits for the ctx's stream, then copies min(iterations run, 1024, capacity) floats to
+ * the HOST array host_out, first iteration first, and writes that count to *n_out.  The ratio of successive entries
+ * estimates the contraction rate of the iteration (the spectral radius of dF/dC near a fixed point).
+ * Returns IDKM_OK, IDKM_ERR_NULL, IDKM_ERR_ORDER (no forward yet), IDKM_ERR_PARAM or IDKM_ERR_CUDA.
+ */
+int idkm_get_history(idkm_ctx* ctx, int which, int layer, float* host_out, int capacity, int* n_out);
+
+/*
  * Whole hot path on HOST buffers (Algorithm 2's per-layer work: cluster, quantise, differentiate):
  * copies W, C0 and dWq to the device, runs idkm_forward_batched and idkm_backward, and copies
  * C, Wq, dW, dC back; returns after everything has completed.  Device buffers are allocated on

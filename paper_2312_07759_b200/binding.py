@@ -63,6 +63,8 @@ lib.idkm_step_noalloc.argtypes = [_fp, C.c_int64, C.c_int, _fp, C.c_int, C.c_flo
 lib.idkm_step_noalloc.restype = C.c_int
 lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
 lib.idkm_set_adjoint_method.restype = C.c_int
+lib.idkm_get_history.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
+lib.idkm_get_history.restype = C.c_int
 lib.idkm_set_forward_loop.argtypes = [_vp, C.c_int]
 lib.idkm_set_forward_loop.restype = C.c_int
 lib.idkm_launch_count.argtypes = [_vp]
@@ -259,6 +261,15 @@ class Context:
     def set_adjoint_method(self, method: int) -> None:
         """0: explicit Jacobian for k*d <= 8 (default); 1: always one fused pass per adjoint step."""
         _check(lib.idkm_set_adjoint_method(self._h, int(method)))
+
+    def history(self, which: int = 0, layer: int = 0, capacity: int = 1024):
+        """``idkm_get_history``: residuals of the last forward (which=0) or implicit backward (which=1) loop of a layer,
+        as a float32 numpy array, first iteration first."""
+        import numpy as np
+        buf = (C.c_float * capacity)()
+        n = C.c_int(0)
+        _check(lib.idkm_get_history(self._h, int(which), int(layer), buf, int(capacity), C.byref(n)))
+        return np.frombuffer(buf, dtype=np.float32, count=n.value).copy()
 
     def set_forward_loop(self, method: int) -> None:
         """0: small layers run the whole forward loop in one cooperative launch (default); 1: a launch per iteration."""

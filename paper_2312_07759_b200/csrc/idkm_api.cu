@@ -130,6 +130,7 @@ static const DualEntry* dual_entry(int d, int k) {
 
 struct WorkspaceLayout {
   size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, off_sync, total;
+  size_t off_hist_fwd, off_hist_adj;
   size_t off_partials64, off_gpartials64, off_gtickets64;   // second set for the fp64 half of the dual step kernel
   int max_slots, max_groups, max_groups64;
 };
@@ -174,6 +175,8 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   w.off_gpartials = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups * plen_max, 256);
   w.off_gtickets = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups, 256);
   w.off_sync = o;      o = align_up(o + 4 * sizeof(unsigned int), 256);   // barrier words of the single-launch loop
+  w.off_hist_fwd = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
+  w.off_hist_adj = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
   const DualEntry* de = dual_entry(d, k);
   const int plen64 = de ? kernel_entry(STEP_PRECISE, d, pick_family(STEP_PRECISE, d, k))->plen : 0;
   w.max_groups64 = de ? w.max_groups : 0;
@@ -290,6 +293,8 @@ static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p)
   p->partials = reinterpret_cast<double*>(ws + wl.off_partials);
   p->gpartials = reinterpret_cast<double*>(ws + wl.off_gpartials);
   p->gtickets = reinterpret_cast<unsigned int*>(ws + wl.off_gtickets);
+  p->hist_fwd = reinterpret_cast<float*>(ws + wl.off_hist_fwd);
+  p->hist_adj = reinterpret_cast<float*>(ws + wl.off_hist_adj);
   p->st = reinterpret_cast<LayerState*>(ws + wl.off_state);
   p->inv_tau = (float)(1.0 / (double)ctx->tau);
   p->inv_tau_d = 1.0 / (double)ctx->tau;
@@ -425,6 +430,7 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   sp.tol = p.tol;
   sp.inv_tau_d = p.inv_tau_d;
   sp.max_iter = max_iter;
+  sp.hist = p.hist_fwd;
   sp.chunked = (m > (long long)SMALL_CHUNK_ROWS * grid * BLOCK) ? 1 : 0;
   sp.spin_limit = SMALL_SPIN_LIMIT;
   // Host-side fault injection for tests of the timeout path (no GPU fault involved: the waits are bounded and the
@@ -756,6 +762,28 @@ int idkm_set_adjoint_method(idkm_ctx* ctx, int method) {
   if (!ctx) return IDKM_ERR_NULL;
   if (method != 0 && method != 1) return IDKM_ERR_PARAM;
   ctx->adjoint_method = method;
+  return IDKM_OK;
+}
+
+int idkm_get_history(idkm_ctx* ctx, int which, int layer, float* host_out, int capacity, int* n_out) {
+  if (!ctx || !host_out || !n_out) return IDKM_ERR_NULL;
+  if (!ctx->have_forward) return IDKM_ERR_ORDER;
+  if ((which != 0 && which != 1) || layer < 0 || layer >= ctx->n_layers || capacity < 0) return IDKM_ERR_PARAM;
+  WorkspaceLayout wl;
+  if (!make_layout(ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+  LayerState st;
+  const char* ws = static_cast<const char*>(ctx->workspace);
+  if (cudaMemcpy(&st, ws + wl.off_state + sizeof(LayerState) * (size_t)layer, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return IDKM_ERR_CUDA;
+  int n = which == 0 ? st.fwd_iters : st.adj_iters;
+  if (n > HIST_CAP) n = HIST_CAP;
+  if (n > capacity) n = capacity;
+  if (n < 0) n = 0;
+  const size_t off = (which == 0 ? wl.off_hist_fwd : wl.off_hist_adj) + sizeof(float) * (size_t)layer * HIST_CAP;
+  if (n > 0 && cudaMemcpy(host_out, ws + off, sizeof(float) * (size_t)n, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return IDKM_ERR_CUDA;
+  *n_out = n;
   return IDKM_OK;
 }
 

@@ -164,6 +164,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
         if (dn < 1e-300) dn = 1e-300;
         res = (float)(sqrt(num) / dn);
         ++it;
+        if (lane == 0 && it <= HIST_CAP) p.hist_adj[(size_t)l * HIST_CAP + it - 1] = res;
         up = (res > prev) ? up + 1 : 0;
         prev = res;
         if (badv > 0.0 || up >= 10) {

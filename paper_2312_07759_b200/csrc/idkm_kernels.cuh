@@ -25,6 +25,7 @@ constexpr float PAD_COORD = 1e18f;   // coordinate of a padding centroid: exp un
 constexpr double S_MIN = 1e-20;      // column sums below this mark a dead cluster
 constexpr float S_MIN_F = 1e-20f;
 constexpr int MAX_BLOCKS_PER_SM = 8;
+constexpr int HIST_CAP = 1024;       // iterations of residual history kept per layer and loop
 // Blocks whose partials one block adds up in the first stage of the cross-block reduction (see finish_layer).
 constexpr int RED_GROUP = 16;
 // Up to this many partials one block adds them all: the extra stage costs a few microseconds of latency, which only
@@ -77,6 +78,8 @@ struct PassParams {
   float* F;           // [L][k][d] F(C_T, W) (FINAL writes)
   float* gvec;        // [L][k][d] direct codebook gradient (GRAD writes)
   float* u;           // [L][k][d] adjoint (GRAD initialises, ADJ updates)
+  float* hist_fwd;    // [L][HIST_CAP]: relative change of C after each forward iteration (first HIST_CAP of them)
+  float* hist_adj;    // [L][HIST_CAP]: relative change of u after each adjoint iteration
   double* partials;   // [(n_blocks + L)][PLEN]
   double* gpartials;  // [(n_blocks + L) / RED_GROUP + L + 2][PLEN]: sums over groups of RED_GROUP partials
   unsigned int* gtickets;   // one arrival counter per group, zero at rest
@@ -415,6 +418,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
       const int it = st->fwd_iters + 1;
       st->fwd_iters = it;
       st->fwd_res = res;
+      if (it <= HIST_CAP) p.hist_fwd[(size_t)l * HIST_CAP + it - 1] = res;
       st->dead = (int)dead;
       if (bad > 0.0) {
         st->status = ST_NONFINITE;
@@ -442,6 +446,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
       const int it = st->adj_iters + 1;
       st->adj_iters = it;
       st->adj_res = res;
+      if (it <= HIST_CAP) p.hist_adj[(size_t)l * HIST_CAP + it - 1] = res;
       const int up = (res > st->adj_prev) ? st->adj_up + 1 : 0;
       st->adj_up = up;
       st->adj_prev = res;
@@ -1336,6 +1341,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_jacobian(const __grid_constant__ P
         if (dn < 1e-300) dn = 1e-300;
         res = (float)(sqrt(num) / dn);
         ++it;
+        if (lane == 0 && it <= HIST_CAP) p.hist_adj[(size_t)l * HIST_CAP + it - 1] = res;
         up = (res > prev) ? up + 1 : 0;
         prev = res;
         if (badv > 0.0 || up >= 10) {
@@ -1498,6 +1504,7 @@ struct SmallLoopParams {
   float tol;
   double inv_tau_d;
   int max_iter;
+  float* hist;           // [HIST_CAP] residual history of the layer
   int chunked;           // 1: some thread has more than 32 rows, fp32 sums are moved out every 32 rows
   int missing_arrivals;  // 0 in production.  Host-side fault injection for the timeout path: the barriers wait for
                          // this many arrivals more than the grid has, so every wait runs out (see idkm.h)

@@ -143,6 +143,9 @@ extern "C" int idkm_step_noalloc(const float* W, int64_t m, int d, const float* 
   p.partials = reinterpret_cast<double*>(nd.scratch + off_part);
   p.gpartials = reinterpret_cast<double*>(nd.scratch + off_gpart);
   p.gtickets = reinterpret_cast<unsigned int*>(nd.scratch + off_gt);
+  // the single step writes one residual: it lands in the unused tail of the 256-byte state area
+  p.hist_fwd = reinterpret_cast<float*>(nd.scratch + 128);
+  p.hist_adj = p.hist_fwd;
   p.inv_tau = (float)(1.0 / (double)tau);
   p.inv_tau_d = 1.0 / (double)tau;
   p.scale = (float)(1.4426950408889634 / (double)tau);

@@ -307,6 +307,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       for (int a = 0; a < D; ++a) c[t][a] = (t < k) ? c_sm[t * D + a] : PAD_COORD;
     iters = it + 1;
     res_f = (float)s_res[0];
+    if (b == 0 && tid == 0 && iters <= HIST_CAP) sp.hist[iters - 1] = res_f;
     dead_n = (int)s_res[1];
     precise = (sqrt(s_res[3]) * sp.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
     if (s_res[2] > 0.0) {

@@ -204,3 +204,46 @@ def test_tiled_explicit_jacobian_on_batched_layers():
         a, b = offs[l], offs[l + 1]
         assert_close(res[0][1][16 * l:16 * (l + 1)], res[1][1][16 * l:16 * (l + 1)], 1e-5, f"dC layer {l}")
         assert_close(res[0][0][a:b], res[1][0][a:b], 1e-5, f"dW layer {l}")
+
+
+@pytest.mark.parametrize("m,d,k,loop,adj", [(3000, 1, 4, 0, 0), (3000, 1, 4, 1, 1), (40000, 2, 16, 0, 0),
+                                            (40000, 2, 16, 1, 1), (60000, 4, 32, 1, 1)])
+def test_residual_history_matches_the_oracle_iteration_by_iteration(m, d, k, loop, adj):
+    """idkm_get_history returns the stop-rule quantity of every iteration: compared with residuals recomputed from the
+    oracle's own iterates (forward: one application of F at a time; adjoint: one application of the adjoint map)."""
+    import torch
+    from oracle import idkm_ref as R
+    from paper_2312_07759_b200 import binding as B
+    T, Ta = 9, 20
+    wl = WL.single_layer(m, d, k, 0.01, std=0.03, seed=3 + k, max_iter=T, adj_max_iter=Ta, g_std=0.5)
+    W, C0, G = (torch.from_numpy(x).cuda() for x in (wl.W, wl.C0, wl.G))
+    ctx = B.Context()
+    ctx.set_forward_loop(loop)
+    ctx.set_adjoint_method(adj)
+    ctx.forward(W, C0, wl.tau, 0.0, T)
+    ctx.backward(G, B.IMPLICIT, 0.0, Ta, 1.0)
+    hf, ha = ctx.history(0), ctx.history(1)
+    info = ctx.info()[0]
+    assert hf.shape == (T,) and ha.shape == (Ta,)
+    assert hf[-1] == np.float32(info.fwd_residual) and ha[-1] == np.float32(info.adj_residual)
+    assert ctx.history(0, capacity=4).shape == (4,)
+    # oracle, iteration by iteration
+    Wd, Gd = wl.W.astype(np.float64), wl.G.astype(np.float64)
+    Cc = wl.C0.astype(np.float64)
+    rf = []
+    for _ in range(T):
+        Cn = R.step(Wd, Cc, wl.tau)[0]
+        rf.append(np.linalg.norm(Cn - Cc) / max(np.linalg.norm(Cn), 1e-300))
+        Cc = Cn
+    assert np.allclose(hf, rf, rtol=2e-3, atol=1e-9)
+    _, _, S, F = R.final(Wd, Cc, wl.tau, want_Wq=False)
+    g = R.codebook_grad(Wd, Gd, Cc, wl.tau)
+    u, ra = g.copy(), []
+    for _ in range(Ta):
+        un = R.adjoint_apply(Wd, Cc, wl.tau, S, F, u) + g
+        ra.append(np.linalg.norm(un - u) / max(np.linalg.norm(un), 1e-300))
+        u = un
+    if d > 1:      # d = 1: the sign kinks make later adjoint residuals differ at the percent level
+        assert np.allclose(ha, ra, rtol=5e-3, atol=1e-9)
+    else:
+        assert np.allclose(ha[:3], ra[:3], rtol=5e-2)
