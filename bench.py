@@ -307,7 +307,7 @@ def main():
     roof["kernel_ms"] = step_kernel_ms
     # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from profiles/step_kernel_cfg4.txt (ncu flushes the
     # caches before the launch, so this is the cold-L2 figure); only known for the profiled workload
-    roof["traffic"] = 67.80e6 + 1.11e6 if wl.name.startswith("cfg4_vq_m4194304") and args.iters == 0 else None
+    roof["traffic"] = 67.21e6 + 0.59e6 if wl.name.startswith("cfg4_vq_m4194304") and args.iters == 0 else None
     roof["roofline_ms"] = max(t_hbm, t_fp32, t_sfu) * 1e3
     # the same two pipes measured now by the library's register-only micro-benchmarks (at the clock of an otherwise
     # idle GPU): the nominal peak above is the contract figure, this one shows how much of it the hardware delivers

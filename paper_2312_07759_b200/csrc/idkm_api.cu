@@ -99,9 +99,10 @@ int pick_family(int mode, int d, int k) {
     const KernelEntry* e = kernel_entry(mode, d, forced);
     if (e && e->launch && e->kpl * e->lpw >= k) return forced;
   }
-  // forward step with more than 128 centroids: the 8-centroids-per-lane, full-warp layout at two blocks per SM
-  // measured 3 % faster than 16 centroids per lane on half-warps
-  if (mode == STEP && k > 128) return N_FAMILY - 1;
+  // forward step with more than 128 centroids: for d <= 2 the 8-centroids-per-lane, full-warp layout at two blocks
+  // per SM is faster than 16 centroids per lane on half-warps (m = 2^22, k = 256: d = 1 0.46 against 0.54 ms, d = 2
+  // 0.71 against 0.77 ms); for d = 4 the half-warp layout wins (0.90 against 0.95 ms)
+  if (mode == STEP && k > 128 && d < 4) return N_FAMILY - 1;
   for (int f = 0; f < N_FAMILY; ++f) {
     const KernelEntry* e = kernel_entry(mode, d, f);
     if (e && e->launch && e->kpl * e->lpw >= k) return f;
