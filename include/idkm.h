@@ -78,7 +78,11 @@ int  idkm_create(idkm_ctx** out);
 void idkm_destroy(idkm_ctx* ctx);
 
 /* Bytes of device workspace the forward and backward need for a problem of m_total rows in
- * n_layers layers (1 for the single-layer calls).  Returns 0 for unsupported d or k. */
+ * n_layers layers (1 for the single-layer calls).  Returns 0 for unsupported d or k.  Besides the
+ * per-layer state and the per-block partial sums it holds, for most codebooks of more than 8
+ * centroids, 8 bytes per row: each row's softmax reference and normaliser, which the codebook-
+ * gradient pass leaves for the adjoint steps (the iteration of Section 4.2 re-evaluates the same attention
+ * rows at every step). */
 size_t idkm_workspace_bytes(int64_t m_total, int d, int k, int n_layers);
 
 /*

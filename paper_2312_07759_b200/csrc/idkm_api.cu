@@ -132,9 +132,12 @@ static const DualEntry* dual_entry(int d, int k) {
 struct WorkspaceLayout {
   size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, off_sync, total;
   size_t off_hist_fwd, off_hist_adj;
+  size_t off_rowstat;   // two floats per weight-vector, or NO_ROWSTAT
   size_t off_partials64, off_gpartials64, off_gtickets64;   // second set for the fp64 half of the dual step kernel
   int max_slots, max_groups, max_groups64;
 };
+
+constexpr size_t NO_ROWSTAT = ~(size_t)0;
 
 static int device_sm_count() {
   int dev = 0, sms = 0;
@@ -146,7 +149,7 @@ static int device_sm_count() {
   return sms;
 }
 
-static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* out) {
+static bool make_layout(int64_t m_total, int d, int k, int n_layers, int sms, WorkspaceLayout* out) {
   if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K || n_layers < 1 || n_layers > IDKM_MAX_LAYERS) return false;
   int plen_max = 1;
   size_t jac_tile_doubles = 0;   // the tiled explicit-Jacobian pass: k d x k d partials, but only two blocks per SM
@@ -184,6 +187,20 @@ static bool make_layout(int d, int k, int n_layers, int sms, WorkspaceLayout* ou
   w.off_partials64 = o;  o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen64, 256);
   w.off_gpartials64 = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups64 * plen64, 256);
   w.off_gtickets64 = o;  o = align_up(o + sizeof(unsigned int) * (size_t)w.max_groups64, 256);
+  // Most group-per-weight adjoint layouts read each row's softmax reference and normaliser, written by the
+  // codebook-gradient pass, instead of recomputing the row minimum and the row sum in every adjoint step.  The two
+  // passes must agree on the layout kind, which they do unless a tuning override forces them apart.
+  const int f_adj = pick_family(ADJ, d, k), f_grad = pick_family(GRAD, d, k);
+  w.off_rowstat = NO_ROWSTAT;
+  if (f_adj >= 0 && f_grad >= 0) {
+    const bool rd = row_cache_layout(d, kernel_entry(ADJ, d, f_adj)->lpw);
+    const bool wr = row_cache_layout(d, kernel_entry(GRAD, d, f_grad)->lpw);
+    if (rd && !wr) return false;
+    if (rd || wr) {
+      w.off_rowstat = o;
+      o = align_up(o + sizeof(float2) * (size_t)m_total, 256);
+    }
+  }
   w.total = o;
   *out = w;
   return true;
@@ -297,6 +314,7 @@ static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p)
   p->hist_fwd = reinterpret_cast<float*>(ws + wl.off_hist_fwd);
   p->hist_adj = reinterpret_cast<float*>(ws + wl.off_hist_adj);
   p->st = reinterpret_cast<LayerState*>(ws + wl.off_state);
+  p->rowstat = (wl.off_rowstat == NO_ROWSTAT) ? nullptr : reinterpret_cast<float2*>(ws + wl.off_rowstat);
   p->inv_tau = (float)(1.0 / (double)ctx->tau);
   p->inv_tau_d = 1.0 / (double)ctx->tau;
   p->scale = (float)(1.4426950408889634 / (double)ctx->tau);
@@ -514,7 +532,7 @@ void idkm_destroy(idkm_ctx* ctx) {
 
 size_t idkm_workspace_bytes(int64_t m_total, int d, int k, int n_layers) {
   WorkspaceLayout wl;
-  if (m_total < 1 || !make_layout(d, k, n_layers, device_sm_count(), &wl)) return 0;
+  if (m_total < 1 || !make_layout(m_total, d, k, n_layers, device_sm_count(), &wl)) return 0;
   return wl.total;
 }
 
@@ -534,7 +552,7 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
       (A_out && !aligned16(A_out)) || (Wq_out && !aligned16(Wq_out)))
     return IDKM_ERR_ALIGN;
   WorkspaceLayout wl;
-  if (!make_layout(d, k, n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (!make_layout(m_total, d, k, n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
   if (workspace_bytes < wl.total) return IDKM_ERR_WORKSPACE;
 
   ctx->have_forward = false;
@@ -605,7 +623,7 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   if (!aligned16(dWq) || (dW_out && !aligned16(dW_out)) || (dC_out && !aligned16(dC_out))) return IDKM_ERR_ALIGN;
   if (dW_out && (dW_out == dWq || dW_out == ctx->W)) return IDKM_ERR_PARAM;
   WorkspaceLayout wl;
-  if (!make_layout(ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (!make_layout(ctx->m_total, ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
   if (workspace_bytes < wl.total) return IDKM_ERR_WORKSPACE;
   ctx->stream = static_cast<cudaStream_t>(cuda_stream);
 
@@ -616,17 +634,21 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   p.max_iter = adj_max_iter;
   p.alpha = alpha;
   ctx->ev_bwd_set = false;
+  const bool solve = (mode == IDKM_IMPLICIT && adj_max_iter > 0);
+  const int fj = pick_family(JACOBIAN, ctx->d, ctx->k);
+  const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, ctx->d, fj)->plen > JAC_SMALL_PLEN_MAX;
+  const bool explicit_jac = ctx->adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS);
+  // the per-row softmax reference and normaliser are kept only if fused adjoint passes follow
+  if (!solve || explicit_jac) p.rowstat = nullptr;
   mark(ctx, 4);
   nvtxRangePushA("idkm codebook gradient");
   int rc = launch_pass(ctx, GRAD, &p, 1);
   nvtxRangePop();
   if (rc != IDKM_OK) return rc;
   mark(ctx, 5);
-  if (mode == IDKM_IMPLICIT && adj_max_iter > 0) {
-    const int fj = pick_family(JACOBIAN, ctx->d, ctx->k);
-    const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, ctx->d, fj)->plen > JAC_SMALL_PLEN_MAX;
+  if (solve) {
     nvtxRangePushA("idkm adjoint solve");
-    if (ctx->adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS))
+    if (explicit_jac)
       rc = launch_pass(ctx, JACOBIAN, &p, 1);      // one pass forms J_C; the whole iteration runs on it in the epilogue
     else
       rc = launch_pass(ctx, ADJ, &p, adj_max_iter);
@@ -655,7 +677,7 @@ int idkm_get_info(idkm_ctx* ctx, idkm_info* info_out) {
   if (!ctx || !info_out) return IDKM_ERR_NULL;
   if (!ctx->have_forward) return IDKM_ERR_ORDER;
   WorkspaceLayout wl;
-  if (!make_layout(ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (!make_layout(ctx->m_total, ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
   LayerState host[MAX_LAYERS];
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
   if (cudaMemcpy(host, static_cast<char*>(ctx->workspace) + wl.off_state, sizeof(LayerState) * (size_t)ctx->n_layers,
@@ -771,7 +793,7 @@ int idkm_get_history(idkm_ctx* ctx, int which, int layer, float* host_out, int c
   if (!ctx->have_forward) return IDKM_ERR_ORDER;
   if ((which != 0 && which != 1) || layer < 0 || layer >= ctx->n_layers || capacity < 0) return IDKM_ERR_PARAM;
   WorkspaceLayout wl;
-  if (!make_layout(ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (!make_layout(ctx->m_total, ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
   if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
   LayerState st;
   const char* ws = static_cast<const char*>(ctx->workspace);

@@ -83,6 +83,8 @@ struct PassParams {
   double* partials;   // [(n_blocks + L)][PLEN]
   double* gpartials;  // [(n_blocks + L) / RED_GROUP + L + 2][PLEN]: sums over groups of RED_GROUP partials
   unsigned int* gtickets;   // one arrival counter per group, zero at rest
+  float2* rowstat;    // [rows] or null: per row the softmax reference (scale * min_j D_ij) and 1 / sum_j exp, as the
+                      // codebook-gradient pass computed them; read by the adjoint layouts of row_cache_layout()
   LayerState* st;
   float inv_tau;      // 1 / tau
   float scale;        // log2(e) / tau
@@ -125,6 +127,11 @@ struct PassCfg {
   static constexpr int MIN_BLOCKS =
       (LPW == 32) ? 2 : ((LPW > 1) ? 1 : ((256 / REGS_EST) > 4 ? 4 : ((256 / REGS_EST) < 1 ? 1 : (256 / REGS_EST))));
 };
+
+// Layouts whose adjoint step reads each row's softmax reference and normaliser from the workspace instead of
+// recomputing them: the group-per-weight layouts, except the full-warp layout at d = 4, whose register budget is
+// full (there the two extra values per row in flight made the step spill and run 8 % slower).
+__host__ __device__ constexpr bool row_cache_layout(int d, int lpw) { return lpw > 1 && !(d == 4 && lpw == 32); }
 
 // ---- special-function-unit wrappers ------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -500,6 +507,11 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   // weight-vectors of a group per unrolled loop body: two in the forward passes (more independent work per warp);
   // one in the backward passes, whose register budget is already full (measured: 4 % faster than two)
   constexpr int WUNROLL = FWD ? 2 : 1;
+  // The adjoint step takes each row's softmax reference and normaliser from p.rowstat (written by the
+  // codebook-gradient pass at the same centroids, with the same arithmetic, so the exponentials come out bit-equal):
+  // no row minimum, no row sum, no cross-lane reduction before the exponentials and no reciprocal.
+  constexpr bool ROWSTAT_R = (MODE == ADJ) && row_cache_layout(D, LPW);
+  constexpr bool ROWSTAT_W = (MODE == GRAD) && row_cache_layout(D, LPW);
 
   // shared: cross-warp reduction buffer (floats), reused by the last block as fp64 scratch
   constexpr int RED_BYTES = ACCUM ? NWARP * PLEN * 4 : 16;
@@ -513,7 +525,8 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   extern __shared__ __align__(16) float slots[];   // [KPL * NA][BLOCK]: second-level sums, one column per thread
   __shared__ __align__(16) float wstage[STAGE];
   __shared__ __align__(16) float gstage[NEED_G ? STAGE : 4];
-  (void)wstage; (void)gstage;
+  __shared__ float2 lstage[ROWSTAT_R ? Cfg::GROUPS * WPG : 1];
+  (void)wstage; (void)gstage; (void)lstage;
 
   const int tid = threadIdx.x;
   const int lane = tid & 31;
@@ -604,7 +617,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   };
 
   // ---- per weight-vector work: returns through the accumulators / writes row outputs ----------
-  auto process = [&](const float (&w)[D], const float (&gi)[D], bool valid, long long row, float (&out)[D]) {
+  auto process = [&](const float (&w)[D], const float (&gi)[D], bool valid, long long row, float (&out)[D], float2 rstat) {
     float dist[KPL];
     float rs[(D > 1 && !FWD) ? KPL : 1];
     (void)rs; (void)dist;
@@ -633,16 +646,28 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
           }
         }
       }
-      lmin = tree_reduce<KPL, 1>(dist);
-      const float gmin = group_min<LPW>(lmin);
-      const float mref = gmin * p.scale;
+      if constexpr (ROWSTAT_R) {
+        // rstat = (reference, 1 / sum) of the row; (0, 0) for a row past the end, which then adds nothing
 #pragma unroll
-      for (int t = 0; t < KPL; ++t) {
-        e[t] = ex2_approx(fmaf(-p.scale, dist[t], mref));
+        for (int t = 0; t < KPL; ++t) e[t] = ex2_approx(fmaf(-p.scale, dist[t], rstat.x));
+        gsum = 1.f;
+        r = rstat.y;
+        (void)lmin; (void)lsum;
+      } else {
+        lmin = tree_reduce<KPL, 1>(dist);
+        const float gmin = group_min<LPW>(lmin);
+        const float mref = gmin * p.scale;
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          e[t] = ex2_approx(fmaf(-p.scale, dist[t], mref));
+        }
+        lsum = tree_reduce<KPL, 0>(e);
+        gsum = group_sum<LPW>(lsum);
+        r = valid ? rcp_approx(gsum) : 0.f;
+        if constexpr (ROWSTAT_W) {
+          if (p.rowstat != nullptr && valid && gl == 0) p.rowstat[row] = make_float2(mref, r);
+        }
       }
-      lsum = tree_reduce<KPL, 0>(e);
-      gsum = group_sum<LPW>(lsum);
-      r = valid ? rcp_approx(gsum) : 0.f;
     }
 
     if constexpr (MODE == STEP || MODE == FINAL) {
@@ -759,8 +784,8 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   };
 
   // rows fetched one tile ahead by this lane (group-per-weight layouts)
-  float pw[LD][D], pg[NEED_G ? LD : 1][D];
-  (void)pw; (void)pg;
+  float pw[LD][D], pg[NEED_G ? LD : 1][D], pl2[ROWSTAT_R ? LD : 1][2];
+  (void)pw; (void)pg; (void)pl2;
   auto fetch = [&](int tl, int ly) {
     if constexpr (LPW > 1) {
       const long long r0 = p.lt.row_off[ly];
@@ -780,6 +805,10 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
             pw[q][0] = x.x; pw[q][1] = x.y;
           } else {
             pw[q][0] = __ldg(p.W + grow);
+          }
+          if constexpr (ROWSTAT_R) {
+            const float2 y = __ldg(p.rowstat + grow);
+            pl2[q][0] = y.x; pl2[q][1] = y.y;
           }
           if constexpr (NEED_G) {
             if constexpr (D == 4) {
@@ -830,6 +859,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
             wstage[(grp * WPG + idx) * D + a] = pw[q][a];
             if constexpr (NEED_G) gstage[(grp * WPG + idx) * D + a] = pg[q][a];
           }
+          if constexpr (ROWSTAT_R) lstage[grp * WPG + idx] = make_float2(pl2[q][0], pl2[q][1]);
         }
       }
       __syncwarp();
@@ -895,8 +925,8 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
           float gdummy[D];
 #pragma unroll
           for (int a = 0; a < D; ++a) gdummy[a] = 0.f;
-          if constexpr (NEED_G) process(wv[un][v], gv[un][v], loc + v < rows, grow + v, outv[v]);
-          else process(wv[un][v], gdummy, loc + v < rows, grow + v, outv[v]);
+          if constexpr (NEED_G) process(wv[un][v], gv[un][v], loc + v < rows, grow + v, outv[v], make_float2(0.f, 0.f));
+          else process(wv[un][v], gdummy, loc + v < rows, grow + v, outv[v], make_float2(0.f, 0.f));
         }
         if constexpr (MODE == FINAL || MODE == SCATTER) {
           float* dst = (MODE == FINAL) ? p.Wq : p.dW;
@@ -951,7 +981,11 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
             gi[0] = gs[0];
           }
         }
-        process(w, gi, ok, grow, outv);
+        float2 rstat = make_float2(0.f, 0.f);
+        if constexpr (ROWSTAT_R) {
+          if (ok) rstat = lstage[grp * WPG + t];
+        }
+        process(w, gi, ok, grow, outv, rstat);
         if constexpr (MODE == FINAL || MODE == SCATTER) {
           float* dst = (MODE == FINAL) ? p.Wq : p.dW;
           if (dst != nullptr && ok && gl == 0) {

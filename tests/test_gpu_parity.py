@@ -169,6 +169,26 @@ def test_batched_unaligned_layer_offsets():
         assert_grad_close(out["dW"][offs[l]:offs[l + 1]], ref["dW"], f"layer {l} dW", nx, TOL_GRAD, TOL_GRAD_KINK)
 
 
+def test_batched_layers_with_row_cached_adjoint():
+    """Ragged batched layers in a group-per-weight layout (k = 24, d = 2): the fused adjoint steps read each row's
+    softmax reference and normaliser, left in the workspace by the codebook-gradient pass, by GLOBAL row index."""
+    rng = np.random.default_rng(11)
+    sizes, d, k = [1001, 530, 2050], 2, 24
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    W = (rng.standard_normal((offs[-1], d)) * 0.03).astype(np.float32)
+    C0 = np.concatenate([W[offs[l]:offs[l + 1]][rng.choice(sizes[l], k, replace=False)] for l in range(3)])
+    G = (rng.standard_normal(W.shape) * 0.5).astype(np.float32)
+    wl = WL.Workload("batched_row_cache", W, C0, G, d, k, float(np.float32(0.012)), 0.0, 10, 0.0, 8, offs, 0)
+    out = gpu_run(wl)
+    assert all(i.status == 0 and i.adj_iters == 8 for i in out["info"])
+    for l, lw in enumerate(WL.split_layers(wl)):
+        ref = oracle_run(lw)
+        a, b = int(offs[l]), int(offs[l + 1])
+        assert_close(out["C"][l * k:(l + 1) * k], ref["C"], TOL_C, f"layer {l} C")
+        assert_close(out["dC"][l * k:(l + 1) * k], ref["dC"], TOL_GRAD, f"layer {l} dC")
+        assert_close(out["dW"][a:b], ref["dW"], TOL_GRAD, f"layer {l} dW")
+
+
 def test_config4_reduced_m_full_k():
     wl = WL.config4(m=1 << 15, iters=20)
     check_workload(wl)
@@ -268,6 +288,7 @@ SWEEP_POINTS = [
     (1 << 20, 4, 1, 0.001), (1 << 20, 4, 4, 0.001), (1 << 20, 4, 8, 0.001),
     (1 << 20, 1, 2, 0.1), (1 << 20, 4, 4, 0.1),            # collapsing: the fp64 step takes over
     (1 << 24, 1, 2, 0.01), (1 << 24, 2, 4, 0.01),
+    (1 << 26, 1, 2, 0.01),                                 # the sweep's largest m
 ]
 
 
