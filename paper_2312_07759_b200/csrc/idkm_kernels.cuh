@@ -131,7 +131,7 @@ struct PassCfg {
 // Layouts whose adjoint step reads each row's softmax reference and normaliser from the workspace instead of
 // recomputing them: the group-per-weight layouts, except the full-warp layout at d = 4, whose register budget is
 // full (there the two extra values per row in flight made the step spill and run 8 % slower).
-__host__ __device__ constexpr bool row_cache_layout(int d, int lpw) { return lpw > 1 && !(d == 4 && lpw == 32); }
+__host__ __device__ constexpr bool row_cache_layout(int d, int lpw) { return lpw > 1; }
 
 // ---- special-function-unit wrappers ------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -526,6 +526,9 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   __shared__ __align__(16) float wstage[STAGE];
   __shared__ __align__(16) float gstage[NEED_G ? STAGE : 4];
   __shared__ float2 lstage[ROWSTAT_R ? Cfg::GROUPS * WPG : 1];
+  __shared__ float2 ostage[ROWSTAT_W ? Cfg::GROUPS * WPG : 1];
+  int stage_slot = 0;   // where the row being processed parks its (reference, 1 / sum)
+  (void)ostage; (void)stage_slot;
   (void)wstage; (void)gstage; (void)lstage;
 
   const int tid = threadIdx.x;
@@ -618,6 +621,56 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
 
   // ---- per weight-vector work: returns through the accumulators / writes row outputs ----------
   auto process = [&](const float (&w)[D], const float (&gi)[D], bool valid, long long row, float (&out)[D], float2 rstat) {
+    if constexpr (ROWSTAT_R) {
+      // Adjoint step with the row's reference and normaliser at hand: nothing separates a pair's distance from its
+      // exponential, so each centroid is taken from distance to eps_ij / (p_ij - pbar_i) in one go and only two
+      // values per centroid (that product's left factor and p_ij) stay live for the second loop.
+      float ers[KPL], z[KPL];
+      float lzp[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        // keeps the shared-memory reads of the second half of the centroids (u_j / S_j, kappa_j) from being hoisted
+        // above the first half's arithmetic, which cost more registers than the full-warp layout at d = 4 has
+        if (US_SMEM && D == 4 && t == KPL / 2) __syncwarp();
+        float dist_t, rs_t = 1.f;
+        if constexpr (D == 1) {
+          dist_t = fabsf(w[0] - c_(t, 0));
+        } else {
+          float sq = 1e-30f;   // rsqrt stays finite when w == c (n_ij = 0 then)
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const float df = w[a] - c_(t, a);
+            sq = fmaf(df, df, sq);
+          }
+          rs_t = rsqrt_approx(sq);
+          dist_t = sq * rs_t;
+        }
+        const float et0 = ex2_approx(fmaf(-p.scale, dist_t, rstat.x));
+        float v = -kap_(t);
+#pragma unroll
+        for (int a = 0; a < D; ++a) v = fmaf(us_(t, a), w[a], v);
+        z[t] = v;
+        lzp[t & 3] = fmaf(et0, v, lzp[t & 3]);
+        ers[t] = (D > 1) ? et0 * rs_t : et0;
+      }
+      const float rr = rstat.y;
+      const float zbar = group_sum<LPW>((lzp[0] + lzp[1]) + (lzp[2] + lzp[3])) * rr;
+      const float rt = rr * p.inv_tau;
+      const float nzr = -zbar * rt;
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        const float et = ers[t] * fmaf(z[t], rt, nzr);   // e_ij(p) / (tau D_ij)
+#pragma unroll
+        for (int a = 0; a < D; ++a) {
+          const float df = w[a] - c_(t, a);
+          float n;
+          if constexpr (D == 1) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
+          else n = df;
+          acc_(t, a) = fmaf(et, n, acc_(t, a));
+        }
+      }
+      return;
+    }
     float dist[KPL];
     float rs[(D > 1 && !FWD) ? KPL : 1];
     (void)rs; (void)dist;
@@ -646,14 +699,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
           }
         }
       }
-      if constexpr (ROWSTAT_R) {
-        // rstat = (reference, 1 / sum) of the row; (0, 0) for a row past the end, which then adds nothing
-#pragma unroll
-        for (int t = 0; t < KPL; ++t) e[t] = ex2_approx(fmaf(-p.scale, dist[t], rstat.x));
-        gsum = 1.f;
-        r = rstat.y;
-        (void)lmin; (void)lsum;
-      } else {
+      {
         lmin = tree_reduce<KPL, 1>(dist);
         const float gmin = group_min<LPW>(lmin);
         const float mref = gmin * p.scale;
@@ -665,7 +711,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         gsum = group_sum<LPW>(lsum);
         r = valid ? rcp_approx(gsum) : 0.f;
         if constexpr (ROWSTAT_W) {
-          if (p.rowstat != nullptr && valid && gl == 0) p.rowstat[row] = make_float2(mref, r);
+          if (gl == 0) ostage[stage_slot] = make_float2(mref, r);   // stored to the workspace once per tile
         }
       }
     }
@@ -985,6 +1031,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         if constexpr (ROWSTAT_R) {
           if (ok) rstat = lstage[grp * WPG + t];
         }
+        if constexpr (ROWSTAT_W) stage_slot = grp * WPG + t;
         process(w, gi, ok, grow, outv, rstat);
         if constexpr (MODE == FINAL || MODE == SCATTER) {
           float* dst = (MODE == FINAL) ? p.Wq : p.dW;
@@ -994,6 +1041,18 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
             else dst[grow] = outv[0];
           }
         }
+      }
+      if constexpr (ROWSTAT_W) {
+        // the tile's (reference, 1 / sum) pairs go to the workspace together, one row per lane
+        __syncwarp();
+        if (p.rowstat != nullptr) {
+#pragma unroll
+          for (int q = 0; q < LD; ++q) {
+            const int idx = gl + q * LPW;
+            if (idx < WPG && gbase + idx < rows) p.rowstat[row0 + gbase + idx] = ostage[grp * WPG + idx];
+          }
+        }
+        __syncwarp();
       }
     }
     if constexpr (ACCUM) {
