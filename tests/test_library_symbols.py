@@ -29,11 +29,12 @@ def test_host_only_calls_work_without_a_device():
     assert "unknown" in B.status_string(12345)
     # larger codebooks need more room for the partial sums
     assert B.workspace_bytes(4096, 4, 256, 1) > B.workspace_bytes(4096, 4, 16, 1)
-    # the row cache of the adjoint step: 8 bytes per row where the adjoint layout uses it (d = 2, k = 256 does,
-    # d = 4, k = 256 and the thread-per-weight layouts of k <= 8 do not)
+    # the row cache of the adjoint step: 8 bytes per row where the adjoint layout is a group-per-weight one (k > 8);
+    # the thread-per-weight layouts of k <= 8 have none
     grow = lambda d, k: B.workspace_bytes(1 << 20, d, k, 1) - B.workspace_bytes(4096, d, k, 1)
     assert grow(2, 256) == 8 * ((1 << 20) - 4096)
-    assert grow(4, 256) == 0 and grow(1, 4) == 0
+    assert grow(4, 256) == 8 * ((1 << 20) - 4096)
+    assert grow(1, 4) == 0 and grow(4, 8) == 0
 
 
 def test_workload_recipes():
