@@ -188,20 +188,32 @@ int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out);
  * cudaFree or other allocating call and needs no idkm_ctx.
  *
  * W [m][d], C_in [k][d], C_out [k][d] are device pointers, 16-byte aligned, owned by the caller; C_in and
- * C_out may alias.  The result is that of idkm_forward with max_iter = 1 (same kernels, same reduction
- * order).  Asynchronous on cuda_stream.
+ * C_out may alias.  The result is that of idkm_forward with max_iter = 1 (same kernels; the cross-block sums
+ * may be grouped differently because this entry point launches at most two blocks per SM).  Asynchronous on
+ * cuda_stream.
  *
- * Limits and sharing.  Returns IDKM_ERR_NOALLOC_TOO_LARGE when (resident blocks + 1) * (1 + 1/16) * padded k
- * * (d+1) * 8 bytes + a few KB exceeds IDKM_NOALLOC_SCRATCH_BYTES; every supported (d, k) fits on a B200, the check
- * guards larger parts.  All calls on a device share the one array, which still holds the previous call's
- * contents when the next begins: the call clears what must start at zero itself, but two calls that
+ * Limits and sharing.  With B = min(2 * SM count, tiles of the layer) blocks and P = padded k * (d+1) doubles
+ * per row of partial sums, the call needs 256 + 1024 + (B + 1) * P * 8 + ((B + 1) / 16 + 3) * P * 8 bytes and
+ * returns IDKM_ERR_NOALLOC_TOO_LARGE when that exceeds IDKM_NOALLOC_SCRATCH_BYTES.  The largest supported
+ * codebook (d = 4, k = 256: P = 1280) needs 3.3 MB on a 148-SM B200, so every supported (d, k) fits there; the
+ * check guards parts with more SMs.  All calls on a device share the one array, which still holds the previous
+ * call's contents when the next begins: the call clears what must start at zero itself, but two calls that
  * overlap on the GPU (different streams, or different host threads) race on it -- serialise them.
  * The first call on each device looks up the array's device address (with that device current) and the
- * SM count; make that first call outside any stream capture.
+ * SM count, under a lock, so concurrent first calls from several host threads are safe; make that first call
+ * outside any stream capture.
  */
 #define IDKM_NOALLOC_SCRATCH_BYTES (4u << 20)
 int idkm_step_noalloc(const float* W, int64_t m, int d, const float* C_in, int k, float tau, float* C_out,
                       void* cuda_stream);
+
+/*
+ * Device-side status of the last idkm_step_noalloc on the current device (the paper has no counterpart).  The step
+ * is asynchronous and has no context to report through: a NaN or Inf in W, C_in or the sums is recorded in the
+ * built-in array.  This call copies that one word to *status_host_out (IDKM_OK or IDKM_ERR_NONFINITE) on
+ * cuda_stream and waits for the stream; it allocates nothing.  Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_CUDA.
+ */
+int idkm_step_noalloc_status(int* status_host_out, void* cuda_stream);
 
 /*
  * How IDKM_IMPLICIT runs the adjoint iteration.  0 (default): where k d <= 64 one pass over W forms the k d x k d
@@ -250,14 +262,30 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
  * adds the partials in the same order and takes the M-step itself, so only the partials cross L2 inside the loop;
  * the loop leaves at the iteration whose stop test passes.  Everything else (batched layers, larger layers or
  * codebooks, max_iter < 2) takes one launch per iteration.  Every barrier wait is bounded (about a second): if one
- * runs out the kernel returns and the layer's status is IDKM_ERR_TIMEOUT.  1: always one launch per iteration.
- * Both run the same iteration; results differ only by the order of the cross-block sums.
- *
- * Test hooks for the timeout path (environment, read at every call; host-side fault injection only -- the waits stay
- * bounded and the kernel returns): IDKM_TEST_MISSING_ARRIVALS=n makes each barrier wait for n arrivals that never
- * come, IDKM_TEST_SPIN_LIMIT=ticks shortens the bound (SM clock ticks).
+ * runs out the kernel returns and the layer's status is IDKM_ERR_TIMEOUT.  1: always one launch per iteration
+ * (for the smallest codebooks -- k <= 4 at d = 1, k <= 2 at d = 2 -- that launch is a kernel that steps the fp32 and
+ * the collapsing, fp64 layers of a batch side by side).  2: as 1, but the fp32 and the fp64 step of an iteration
+ * are always two launches, one after the other.  All three run the same iteration; 0 differs from the others only by
+ * the order of the cross-block sums, 1 and 2 give bitwise the same result.
  */
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
+
+/*
+ * Host-side fault injection for tests of the timeout path of the one-launch forward loop (no GPU fault is involved:
+ * the waits stay bounded and the kernel returns).  missing_arrivals = n > 0 makes each grid-wide barrier of this
+ * ctx's following calls wait for n arrivals that never come; spin_limit_ticks > 0 shortens the bound of every wait
+ * to that many SM clock ticks.  (0, 0) restores production behaviour, which is also the state after idkm_create.
+ * Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_PARAM (a negative argument).
+ */
+int idkm_set_test_hooks(idkm_ctx* ctx, int missing_arrivals, int64_t spin_limit_ticks);
+
+/*
+ * Consistency self-check: waits for the ctx's stream and counts the arrival counters of the cross-block reductions
+ * in the last forward's workspace that are not at rest.  Every counter returns to zero when its reduction
+ * completes, so *count_out (HOST) is 0 after any completed call; anything else means a reduction was entered by
+ * some blocks and never finished.  Returns IDKM_OK, IDKM_ERR_NULL, IDKM_ERR_ORDER (no forward yet) or IDKM_ERR_CUDA.
+ */
+int idkm_count_busy_tickets(idkm_ctx* ctx, int* count_out);
 
 /* Number of kernels this ctx has launched since idkm_create (for accounting in benchmarks). */
 int64_t idkm_launch_count(const idkm_ctx* ctx);

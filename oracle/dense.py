@@ -14,36 +14,41 @@ from __future__ import annotations
 import numpy as np
 
 
-def attention(W: np.ndarray, C: np.ndarray, tau: float):
-    """A = rowsoftmax_tau(-D), D_ij = ||w_i - c_j||; also returns D and the unit vectors n_ij."""
+def attention(W: np.ndarray, C: np.ndarray, tau: float, squared: bool = False):
+    """A = rowsoftmax_tau(-D), D_ij = ||w_i - c_j|| (squared: ||w_i - c_j||^2, the variant in which the objectives
+    of Sections 3.1 / 3.2 are written); also returns D and n_ij = dD_ij/dw_i (unit vectors; squared: 2 (w_i - c_j))."""
     diff = W[:, None, :] - C[None, :, :]                  # [m, k, d]
-    D = np.sqrt((diff ** 2).sum(-1))                      # [m, k]
+    D2 = (diff ** 2).sum(-1)                              # [m, k]
+    D = D2 if squared else np.sqrt(D2)
     X = -(D - D.min(axis=1, keepdims=True)) / tau
     E = np.exp(X)
     A = E / E.sum(axis=1, keepdims=True)
-    with np.errstate(invalid="ignore", divide="ignore"):
-        n = np.where(D[..., None] > 0, diff / D[..., None], 0.0)
+    if squared:
+        n = 2.0 * diff
+    else:
+        with np.errstate(invalid="ignore", divide="ignore"):
+            n = np.where(D[..., None] > 0, diff / D[..., None], 0.0)
     return A, D, n
 
 
-def fixed_point_map(W, C, tau):
+def fixed_point_map(W, C, tau, squared: bool = False):
     """F(C, W)_j = sum_i A_ij w_i / sum_i A_ij."""
-    A, _, _ = attention(W, C, tau)
+    A, _, _ = attention(W, C, tau, squared)
     S = A.sum(0)
     return (A.T @ W) / S[:, None], S, A
 
 
-def soft_quantise(W, C, tau):
+def soft_quantise(W, C, tau, squared: bool = False):
     """Wq = A C."""
-    A, _, _ = attention(W, C, tau)
+    A, _, _ = attention(W, C, tau, squared)
     return A @ C
 
 
-def jacobians(W: np.ndarray, C: np.ndarray, tau: float):
+def jacobians(W: np.ndarray, C: np.ndarray, tau: float, squared: bool = False):
     """Explicit J_C = dF/dC [kd, kd], dF/dW [kd, md], dWq/dC [md, kd], dWq/dW [md, md] at (C, W)."""
     m, d = W.shape
     k = C.shape[0]
-    A, D, n = attention(W, C, tau)
+    A, D, n = attention(W, C, tau, squared)
     S = A.sum(0)
     F = (A.T @ W) / S[:, None]
     eye_k = np.eye(k)
@@ -70,13 +75,13 @@ def jacobians(W: np.ndarray, C: np.ndarray, tau: float):
     return J_C, dF_dW, dWq_dC, dWq_dW.reshape(m * d, m * d), S, F
 
 
-def gradients(W, G, C, tau, mode="implicit"):
+def gradients(W, G, C, tau, mode="implicit", squared: bool = False):
     """(dL/dW [m, d], u [k, d]) of L = <G, Wq(W, C*(W))> with the linear system solved exactly.
 
     implicit: u = (I - J_C^T)^-1 g;  jfb: u = g  (zeroth Neumann term, Section 4.3)."""
     m, d = W.shape
     k = C.shape[0]
-    J_C, dF_dW, dWq_dC, dWq_dW, _, _ = jacobians(W, C, tau)
+    J_C, dF_dW, dWq_dC, dWq_dW, _, _ = jacobians(W, C, tau, squared)
     gflat = G.reshape(-1)
     g = dWq_dC.T @ gflat
     if mode == "implicit":

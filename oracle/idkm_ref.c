@@ -25,6 +25,12 @@
  *     (u* = M*^T g); zero adjoint iterations is Jacobian-free backprop (M* = I);
  *   - dL/dC output := u.
  *
+ * Variant (idkm_ref_set_squared(1)): the softmax takes the SQUARED distance, D_ij = ||w_i - c_j||^2, the quantity
+ * the clustering objectives are written in (Section 3.1, the k-means objective; Section 3.2, the soft objective that
+ * the iteration is derived from).  Everything below is written in terms of D_ij and its gradient
+ * n_ij = dD_ij/dw_i = -dD_ij/dc_j, so the variant changes two lines: D_ij itself and n_ij = 2 (w_i - c_j), which has
+ * no kink.  The method as published (Algorithm 1, step 3) is the default.
+ *
  * Sums over i run in NCHUNK fixed row chunks (so that OpenMP may take one chunk per thread)
  * and the chunk sums are added in chunk order: the result does not depend on the thread count.
  * Nothing else is blocked, fused or reordered.
@@ -56,6 +62,12 @@ void idkm_ref_set_threads(int n) {
 #endif
 }
 
+/* 0: D_ij is the Euclidean norm (Algorithm 1, step 3).  1: its square (the variant described above). */
+static int g_squared = 0;
+
+void idkm_ref_set_squared(int on) { g_squared = (on != 0); }
+int idkm_ref_get_squared(void) { return g_squared; }
+
 static void chunk_bounds(int64_t m, int c, int64_t *lo, int64_t *hi) {
   *lo = (m * (int64_t)c) / NCHUNK;
   *hi = (m * (int64_t)(c + 1)) / NCHUNK;
@@ -72,7 +84,7 @@ static void attention_row(const double *w, const double *C, int k, int d, double
       double t = w[a] - C[(int64_t)j * d + a];
       s += t * t;
     }
-    D[j] = sqrt(s);
+    D[j] = g_squared ? s : sqrt(s);
     if (D[j] < dmin) dmin = D[j];
   }
   double sum = 0.0;
@@ -83,8 +95,12 @@ static void attention_row(const double *w, const double *C, int k, int d, double
   for (int j = 0; j < k; ++j) A[j] /= sum;
 }
 
-/* n_ij = (w_i - c_j) / D_ij, zero vector when D_ij == 0. */
+/* n_ij = dD_ij/dw_i: the unit vector (w_i - c_j) / D_ij, zero when D_ij == 0; for the squared distance 2 (w_i - c_j). */
 static void unit_vector(const double *w, const double *cj, double Dj, int d, double *n) {
+  if (g_squared) {
+    for (int a = 0; a < d; ++a) n[a] = 2.0 * (w[a] - cj[a]);
+    return;
+  }
   for (int a = 0; a < d; ++a) n[a] = (Dj > 0.0) ? (w[a] - cj[a]) / Dj : 0.0;
 }
 

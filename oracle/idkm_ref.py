@@ -51,6 +51,34 @@ def set_threads(n: int) -> None:
     _L().idkm_ref_set_threads(C.c_int(n))
 
 
+def set_squared(on: bool) -> None:
+    """Switches the softmax to the squared distance D_ij = ||w_i - c_j||^2 (the variant in which the objectives of
+    Sections 3.1 / 3.2 are written); off is the method as published."""
+    _L().idkm_ref_set_squared(C.c_int(1 if on else 0))
+
+
+def get_squared() -> bool:
+    lib = _L()
+    lib.idkm_ref_get_squared.restype = C.c_int
+    return bool(lib.idkm_ref_get_squared())
+
+
+class squared_distance:
+    """``with squared_distance():`` runs the enclosed oracle calls with the squared-distance softmax."""
+
+    def __init__(self, on: bool = True):
+        self.on = on
+
+    def __enter__(self):
+        self.prev = get_squared()
+        set_squared(self.on)
+        return self
+
+    def __exit__(self, *exc):
+        set_squared(self.prev)
+        return False
+
+
 def _f64(x) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(x, dtype=np.float64))
 

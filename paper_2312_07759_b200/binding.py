@@ -61,6 +61,12 @@ lib.idkm_get_phase_ms.argtypes = [_vp, C.POINTER(C.c_float)]
 lib.idkm_get_phase_ms.restype = C.c_int
 lib.idkm_step_noalloc.argtypes = [_fp, C.c_int64, C.c_int, _fp, C.c_int, C.c_float, _fp, _vp]
 lib.idkm_step_noalloc.restype = C.c_int
+lib.idkm_step_noalloc_status.argtypes = [C.POINTER(C.c_int), _vp]
+lib.idkm_step_noalloc_status.restype = C.c_int
+lib.idkm_set_test_hooks.argtypes = [_vp, C.c_int, C.c_int64]
+lib.idkm_set_test_hooks.restype = C.c_int
+lib.idkm_count_busy_tickets.argtypes = [_vp, C.POINTER(C.c_int)]
+lib.idkm_count_busy_tickets.restype = C.c_int
 lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
 lib.idkm_set_adjoint_method.restype = C.c_int
 lib.idkm_get_history.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
@@ -129,6 +135,13 @@ def step_noalloc(W, C_in, tau: float, C_out=None, stream=None):
     _check(lib.idkm_step_noalloc(_ptr(W), int(W.shape[0]), int(W.shape[1]), _ptr(C_in), int(C_in.shape[0]),
                                  float(tau), _ptr(C_out), _stream(stream)))
     return C_out
+
+
+def step_noalloc_status(stream=None) -> int:
+    """``idkm_step_noalloc_status``: the device-side status of the last ``step_noalloc`` on the current device."""
+    st = C.c_int(0)
+    _check(lib.idkm_step_noalloc_status(C.byref(st), _stream(stream)))
+    return int(st.value)
 
 
 def assign(W, Cm, want_codes: bool = True, want_Wq: bool = True, stream=None):
@@ -272,8 +285,19 @@ class Context:
         return np.frombuffer(buf, dtype=np.float32, count=n.value).copy()
 
     def set_forward_loop(self, method: int) -> None:
-        """0: small layers run the whole forward loop in one cooperative launch (default); 1: a launch per iteration."""
+        """0: small layers run the whole forward loop in one cooperative launch (default); 1: a launch per iteration;
+        2: a launch per iteration and never the kernel that steps fp32 and fp64 layers side by side."""
         _check(lib.idkm_set_forward_loop(self._h, int(method)))
+
+    def set_test_hooks(self, missing_arrivals: int = 0, spin_limit_ticks: int = 0) -> None:
+        """``idkm_set_test_hooks``: host-side fault injection for the timeout path; (0, 0) switches it off."""
+        _check(lib.idkm_set_test_hooks(self._h, int(missing_arrivals), int(spin_limit_ticks)))
+
+    def busy_tickets(self) -> int:
+        """``idkm_count_busy_tickets``: arrival counters of the last forward's workspace that are not at rest."""
+        n = C.c_int(0)
+        _check(lib.idkm_count_busy_tickets(self._h, C.byref(n)))
+        return int(n.value)
 
     def set_timing(self, enable: bool = True) -> None:
         _check(lib.idkm_set_timing(self._h, 1 if enable else 0))

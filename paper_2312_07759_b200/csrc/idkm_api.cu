@@ -38,7 +38,7 @@ __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0,
     s.fwd_done = 0; s.fwd_iters = 0; s.fwd_res = 0.f; s.dead = 0;
     s.adj_done = 0; s.adj_iters = 0; s.adj_res = 0.f; s.status = ST_OK;
     s.ticket = 0u; s.adj_up = 0; s.adj_prev = 3.0e38f;
-    for (int q = 0; q < 4; ++q) s.pad[q] = 0;
+    for (int q = 0; q < 3; ++q) s.pad[q] = 0;
     // bounding box of the starting centroids decides which step kernel takes the layer first
     double box2 = 0.0;
     for (int a = 0; a < d; ++a) {
@@ -50,7 +50,7 @@ __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0,
       }
       box2 += (hi - lo) * (hi - lo);
     }
-    s.precise = (sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
+    s.precise[0] = s.precise[1] = (sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
     st[i] = s;
   }
   if (C0 != C)
@@ -233,7 +233,10 @@ struct idkm_ctx {
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
-  int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never
+  int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never;
+                        // 2: never, and the fp32 and fp64 steps of an iteration are always two launches
+  int hook_missing_arrivals;      // host-side fault injection for the timeout path (idkm_set_test_hooks); 0 at rest
+  long long hook_spin_limit;      // 0: the default bound
   int small_blocks[3][N_SMALL_FAMILY];   // cached co-resident grid of the single-launch loop kernels (0 = not queried)
   // bounded run-ahead of the tolerance-mode loops: a pinned host word the device sets when all layers are done
   int* h_flag;
@@ -362,7 +365,7 @@ static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams
   const KernelEntry* e32 = kernel_entry(STEP, ctx->d, f32);
   const KernelEntry* e64 = kernel_entry(STEP_PRECISE, ctx->d, f64);
   static const bool dual_off = (getenv("IDKM_NO_DUAL") != nullptr);   // tuning knob: always two launches per iteration
-  const DualEntry* de = dual_off ? nullptr : dual_entry(ctx->d, ctx->k);
+  const DualEntry* de = (dual_off || ctx->forward_loop == 2) ? nullptr : dual_entry(ctx->d, ctx->k);
   PassParams q = *p;
   int rc = build_table(ctx, STEP, f32, &p->lt);
   if (rc != IDKM_OK) return rc;
@@ -452,14 +455,10 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   sp.hist = p.hist_fwd;
   sp.chunked = (m > (long long)SMALL_CHUNK_ROWS * grid * BLOCK) ? 1 : 0;
   sp.spin_limit = SMALL_SPIN_LIMIT;
-  // Host-side fault injection for tests of the timeout path (no GPU fault involved: the waits are bounded and the
-  // kernel returns): IDKM_TEST_MISSING_ARRIVALS=n makes every barrier wait for n arrivals that never come,
-  // IDKM_TEST_SPIN_LIMIT=ticks shortens the wait.  Both are read per call.
-  if (const char* e = getenv("IDKM_TEST_MISSING_ARRIVALS")) sp.missing_arrivals = atoi(e) > 0 ? atoi(e) : 0;
-  if (const char* e = getenv("IDKM_TEST_SPIN_LIMIT")) {
-    const long long v = atoll(e);
-    if (v > 0 && v < SMALL_SPIN_LIMIT) sp.spin_limit = v;
-  }
+  // Host-side fault injection for tests of the timeout path (idkm_set_test_hooks; no GPU fault involved: the waits
+  // are bounded and the kernel returns)
+  sp.missing_arrivals = ctx->hook_missing_arrivals;
+  if (ctx->hook_spin_limit > 0 && ctx->hook_spin_limit < SMALL_SPIN_LIMIT) sp.spin_limit = ctx->hook_spin_limit;
   if (se->launch(sp, (int)grid, ctx->stream) != cudaSuccess) {
     (void)cudaGetLastError();
     return 1;   // nothing was queued: take the launch-per-iteration path
@@ -812,8 +811,44 @@ int idkm_get_history(idkm_ctx* ctx, int which, int layer, float* host_out, int c
 
 int idkm_set_forward_loop(idkm_ctx* ctx, int method) {
   if (!ctx) return IDKM_ERR_NULL;
-  if (method != 0 && method != 1) return IDKM_ERR_PARAM;
+  if (method < 0 || method > 2) return IDKM_ERR_PARAM;
   ctx->forward_loop = method;
+  return IDKM_OK;
+}
+
+int idkm_set_test_hooks(idkm_ctx* ctx, int missing_arrivals, int64_t spin_limit_ticks) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (missing_arrivals < 0 || spin_limit_ticks < 0) return IDKM_ERR_PARAM;
+  ctx->hook_missing_arrivals = missing_arrivals;
+  ctx->hook_spin_limit = spin_limit_ticks;
+  return IDKM_OK;
+}
+
+int idkm_count_busy_tickets(idkm_ctx* ctx, int* count_out) {
+  if (!ctx || !count_out) return IDKM_ERR_NULL;
+  if (!ctx->have_forward) return IDKM_ERR_ORDER;
+  WorkspaceLayout wl;
+  if (!make_layout(ctx->m_total, ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+  const char* ws = static_cast<const char*>(ctx->workspace);
+  int busy = 0;
+  LayerState host[MAX_LAYERS];
+  if (cudaMemcpy(host, ws + wl.off_state, sizeof(LayerState) * (size_t)ctx->n_layers, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return IDKM_ERR_CUDA;
+  for (int l = 0; l < ctx->n_layers; ++l) busy += (host[l].ticket != 0u);
+  const size_t offs[2] = {wl.off_gtickets, wl.off_gtickets64};
+  const int counts[2] = {wl.max_groups, wl.max_groups64};
+  for (int s = 0; s < 2; ++s) {
+    if (counts[s] <= 0) continue;
+    unsigned int* t = new (std::nothrow) unsigned int[counts[s]];
+    if (!t) return IDKM_ERR_CUDA;
+    const cudaError_t rc = cudaMemcpy(t, ws + offs[s], sizeof(unsigned int) * (size_t)counts[s], cudaMemcpyDeviceToHost);
+    if (rc == cudaSuccess)
+      for (int i = 0; i < counts[s]; ++i) busy += (t[i] != 0u);
+    delete[] t;
+    if (rc != cudaSuccess) return IDKM_ERR_CUDA;
+  }
+  *count_out = busy;
   return IDKM_OK;
 }
 

@@ -52,9 +52,12 @@ struct LayerState {   // 64 bytes, one per layer, in the workspace
   unsigned int ticket;
   int adj_up;        // consecutive adjoint steps whose residual grew
   float adj_prev;
-  int precise;       // 1: the layer's centroids lie within PRECISE_SPAN * tau of each other (collapsing); the
-                     // forward step then runs in the fp64 kernel
-  int pad[4];
+  int precise[2];    // [t & 1] routes forward iteration t.  1: the layer's centroids lie within PRECISE_SPAN * tau of
+                     // each other (collapsing) and the step runs in the fp64 kernel.  The epilogue of iteration t
+                     // writes entry (t + 1) & 1 only, so nothing a launch routes by changes while it runs: the fp32
+                     // and the fp64 half of the dual step kernel, whose blocks are not ordered against each other,
+                     // can never both take (or both skip) a layer.
+  int pad[3];
 };
 static_assert(sizeof(LayerState) == 64, "LayerState layout");
 
@@ -418,7 +421,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   if (tid == 0) {
     st->ticket = 0u;
     if constexpr (MODE == STEP) {
-      st->precise = (sqrt(box2) * p.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
+      st->precise[(p.iter + 1) & 1] = (sqrt(box2) * p.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
       double dn = sqrt(den);
       if (dn < 1e-300) dn = 1e-300;
       const float res = (float)(sqrt(num) / dn);
@@ -885,7 +888,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
       if (cur_layer >= 0 && layer_active) flush(cur_layer);
       cur_layer = layer;
       if constexpr (MODE == STEP)
-        layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise == 0) && (p.st[layer].fwd_iters == p.iter);
+        layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[p.iter & 1] == 0) && (p.st[layer].fwd_iters == p.iter);
       else if constexpr (MODE == ADJ) layer_active = (p.st[layer].adj_done == 0);
       else layer_active = true;
       if constexpr (US_SMEM) __syncthreads();   // the previous layer's table is no longer read
@@ -1188,7 +1191,7 @@ __device__ __forceinline__ void precise_body(const PassParams& p) {
     if (layer != cur_layer) {
       if (cur_layer >= 0 && layer_active) flush(cur_layer);
       cur_layer = layer;
-      layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise != 0) && (p.st[layer].fwd_iters == p.iter);
+      layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[p.iter & 1] != 0) && (p.st[layer].fwd_iters == p.iter);
       if (layer_active) {
         const float* Cl = p.C + (size_t)layer * k * D;
 #pragma unroll

@@ -12,6 +12,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "../../include/idkm.h"
 
 namespace idkm {
@@ -22,12 +24,39 @@ constexpr size_t NOALLOC_SCRATCH_BYTES = IDKM_NOALLOC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
 constexpr int NOALLOC_MAX_DEVICES = 64;
+// Resident blocks per SM this entry point launches at most.  The partial-sum rows of the largest codebook
+// (d = 4, k = 256: 10 KB each) times (blocks + 1), plus the group rows, must fit the fixed array: two blocks per SM
+// on a 148-SM part need 3.3 MB of the 4 MiB, whatever register count the compiler gives the kernels.
+constexpr int NOALLOC_BLOCKS_PER_SM = 2;
 struct NoallocDevice {
   bool ready;
   unsigned char* scratch;   // DEVICE address of g_noalloc_scratch on that device
   int sms;
 };
 static NoallocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+static std::mutex g_noalloc_mu;   // guards the table above: two host threads may make their first call together
+
+// Looks up (once per device, with that device current) the device address of the built-in array and the SM count.
+static int noalloc_device(NoallocDevice* out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return IDKM_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  NoallocDevice& nd = g_noalloc_dev[dev];
+  if (!nd.ready) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+      (void)cudaGetLastError();
+      return IDKM_ERR_CUDA;
+    }
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return IDKM_ERR_CUDA;
+    nd.scratch = static_cast<unsigned char*>(ptr);
+    nd.sms = sms;
+    nd.ready = true;
+  }
+  *out = nd;
+  return IDKM_OK;
+}
 
 // Resets the single layer's state and seeds C_out with the starting centroids.  The scratch keeps
 // whatever the previous call left, so everything the step reads before writing is set here.
@@ -50,7 +79,7 @@ __global__ void idkm_noalloc_init(LayerState* st, const float* C_in, float* C_ou
       }
       box2 += (hi - lo) * (hi - lo);
     }
-    s.precise = (sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
+    s.precise[0] = s.precise[1] = (sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
     *st = s;
   }
   if (C_in != C_out)
@@ -76,7 +105,7 @@ static int noalloc_table(const KernelEntry* e, int64_t m, int sms, LayerTable* l
     (void)cudaGetLastError();
     per_sm = 1;
   }
-  if (per_sm > MAX_BLOCKS_PER_SM) per_sm = MAX_BLOCKS_PER_SM;
+  if (per_sm > NOALLOC_BLOCKS_PER_SM) per_sm = NOALLOC_BLOCKS_PER_SM;
   long long nb = (long long)sms * per_sm;
   if (nb > tiles) nb = tiles;
   lt->n_blocks = (int)nb;
@@ -96,21 +125,9 @@ extern "C" int idkm_step_noalloc(const float* W, int64_t m, int d, const float* 
   if (((uintptr_t)W | (uintptr_t)C_in | (uintptr_t)C_out) & 15u) return IDKM_ERR_ALIGN;
 
   // once per device, with that device current: turn the symbol into a device address
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return IDKM_ERR_CUDA;
-  NoallocDevice& nd = g_noalloc_dev[dev];
-  if (!nd.ready) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
-      (void)cudaGetLastError();
-      return IDKM_ERR_CUDA;
-    }
-    int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return IDKM_ERR_CUDA;
-    nd.scratch = static_cast<unsigned char*>(ptr);
-    nd.sms = sms;
-    nd.ready = true;
-  }
+  NoallocDevice nd;
+  const int rc_dev = noalloc_device(&nd);
+  if (rc_dev != IDKM_OK) return rc_dev;
 
   const int f32 = pick_family(STEP, d, k), f64 = pick_family(STEP_PRECISE, d, k);
   if (f32 < 0 || f64 < 0) return IDKM_ERR_UNSUPPORTED;
@@ -131,6 +148,7 @@ extern "C" int idkm_step_noalloc(const float* W, int64_t m, int d, const float* 
   const int nb_max = p.lt.n_blocks > lt64.n_blocks ? p.lt.n_blocks : lt64.n_blocks;
   const int plen_max = e32->plen > e64->plen ? e32->plen : e64->plen;
   const int n_groups = (nb_max + 1) / RED_GROUP + 3;
+  // bytes: 256 (state) + 1024 (group counters) + (nb_max + 1) partial rows + n_groups group rows of plen_max doubles
   const size_t off_gt = 256, off_part = off_gt + 1024;
   const size_t off_gpart = off_part + sizeof(double) * (size_t)(nb_max + 1) * plen_max;
   const size_t need = off_gpart + sizeof(double) * (size_t)n_groups * plen_max;
@@ -161,5 +179,24 @@ extern "C" int idkm_step_noalloc(const float* W, int64_t m, int d, const float* 
   if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
   if (e32->launch(p, p.lt.n_blocks, stream) != cudaSuccess) return IDKM_ERR_CUDA;
   if (e64->launch(q, q.lt.n_blocks, stream) != cudaSuccess) return IDKM_ERR_CUDA;
+  return IDKM_OK;
+}
+
+// The status word the last idkm_step_noalloc on this device left in the built-in array (IDKM_OK, or
+// IDKM_ERR_NONFINITE when W, C_in or the sums held a NaN / Inf): one 4-byte copy to the host, no allocation.
+extern "C" int idkm_step_noalloc_status(int* status_host_out, void* cuda_stream) {
+  if (!status_host_out) return IDKM_ERR_NULL;
+  NoallocDevice nd;
+  const int rc_dev = noalloc_device(&nd);
+  if (rc_dev != IDKM_OK) return rc_dev;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const LayerState* st = reinterpret_cast<const LayerState*>(nd.scratch);
+  int status = 0;
+  if (cudaMemcpyAsync(&status, &st->status, sizeof(int), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return IDKM_ERR_CUDA;
+  }
+  *status_host_out = status;
   return IDKM_OK;
 }

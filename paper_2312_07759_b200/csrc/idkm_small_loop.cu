@@ -68,7 +68,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
 
   // uniform loop state (identical in every thread of every block)
   int iters = 0, done = 0, status = ST_OK, dead_n = 0;
-  int precise = sp.st[0].precise;
+  int precise = sp.st[0].precise[0];
   float res_f = 0.f;
   if (tid < k * D) c_sm[tid] = sp.C[tid];
   __syncthreads();
@@ -330,7 +330,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       st->fwd_res = res_f;
       st->dead = dead_n;
       st->fwd_done = done;
-      st->precise = precise;
+      st->precise[0] = st->precise[1] = precise;
       st->status = ok ? status : ST_TIMEOUT;
       st->ticket = 0u;
     }

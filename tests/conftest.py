@@ -24,3 +24,16 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    """Writes the achieved parity errors the GPU tests recorded to the file IDKM_PARITY_TABLE names, if any."""
+    path = os.environ.get("IDKM_PARITY_TABLE")
+    if not path:
+        return
+    try:
+        import parity_util
+    except Exception:
+        return
+    if parity_util.RECORDS:
+        parity_util.write_records(path)

@@ -3,7 +3,7 @@ import numpy as np
 import pytest
 
 from paper_2312_07759_b200 import workloads as WL
-from parity_util import TOL_C, TOL_GRAD, assert_close, oracle_run
+from parity_util import TOL_C, TOL_GRAD, assert_close, at_centroids, oracle_backward_at, oracle_run
 
 pytestmark = pytest.mark.gpu
 
@@ -122,22 +122,52 @@ def test_explicit_jacobian_adjoint_equals_fused_passes(m, d, k):
     assert abs(res[0][2] - res[1][2]) <= 1e-3 * max(res[1][2], 1e-30) + 1e-9
     assert abs(res[(0, "tol")][0] - res[(1, "tol")][0]) <= 1
     assert_close(res[(0, "tol")][1], res[(1, "tol")][1], 1e-3, "dC at tolerance")
+    # against the oracle at common centroids (the oracle's, handed over with the loop switched off): the gradient
+    # tolerance for every d, scalar weights included -- no weight can lie between two identical centroid sets
     ref = oracle_run(wl)
-    assert_close(res[0][1], ref["dC"], TOL_GRAD if d > 1 else 3e-2, "dC vs oracle")
+    wc = at_centroids(wl, ref["C"])
+    refc = oracle_backward_at(wc, wc.C0)
+    for method in (0, 1):
+        ctx = B.Context()
+        ctx.set_adjoint_method(method)
+        ctx.forward(torch.from_numpy(wc.W).cuda(), torch.from_numpy(wc.C0).cuda(), wc.tau, 0.0, 0)
+        dWc, dCc = ctx.backward(G, B.IMPLICIT, 0.0, wl.adj_max_iter, 1.0)
+        assert_close(dCc.cpu().numpy(), refc["dC"], TOL_GRAD, f"dC vs oracle at common C, adjoint method {method}")
+        assert_close(dWc.cpu().numpy(), refc["dW"], TOL_GRAD, f"dW vs oracle at common C, adjoint method {method}")
 
 
 def test_pipe_rate_microbenchmarks():
-    """The measured fp32 and special-function issue rates land near the documented widths of the two pipes
-    (128 and 16 results per clock per SM): between 60 % and 105 % of width x SM count x maximum SM clock (a
-    lower clock under load or a power cap lowers the figure, nothing raises it)."""
+    """The measured fp32 and special-function issue rates are positive, stand in the ratio of the two pipes' widths
+    (128 : 16 results per clock per SM) and, divided by the SM clock read (never set) through NVML around the
+    measurement, land near those widths.  The clock of a shared GPU is whatever it is, so nothing here depends on
+    the part's maximum clock."""
     import torch
     from paper_2312_07759_b200 import binding as B
-    props = torch.cuda.get_device_properties(0)
-    sms = props.multi_processor_count
-    clk_hz = 1965e6                   # maximum SM clock of the part
-    fp32, sfu = B.measure_pipe_rates()
-    assert 0.60 < fp32 / (sms * 128 * clk_hz) < 1.05, fp32
-    assert 0.60 < sfu / (sms * 16 * clk_hz) < 1.05, sfu
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    clocks = []
+    try:
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(torch.cuda.current_device())
+        read_clock = lambda: float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+    except Exception:
+        read_clock = None
+    B.measure_pipe_rates()                      # brings the clock up before it is read
+    fp32 = sfu = 0.0
+    for _ in range(3):
+        if read_clock:
+            clocks.append(read_clock())
+        a, b = B.measure_pipe_rates()
+        fp32, sfu = max(fp32, a), max(sfu, b)
+        if read_clock:
+            clocks.append(read_clock())
+    assert fp32 > 0 and sfu > 0
+    assert 6.0 < fp32 / sfu < 10.0, (fp32, sfu)
+    if clocks:
+        # the highest clock seen bounds the rate from above, the lowest from below (the clock may move in between)
+        hi, lo = max(clocks) * 1e6, min(clocks) * 1e6
+        assert fp32 / (sms * 128 * hi) < 1.10 and fp32 / (sms * 128 * lo) > 0.50, (fp32, clocks)
+        assert sfu / (sms * 16 * hi) < 1.10 and sfu / (sms * 16 * lo) > 0.50, (sfu, clocks)
     assert B.lib.idkm_measure_pipe_rates(None, None, None) == B.ERR_NULL
 
 
@@ -247,3 +277,43 @@ def test_residual_history_matches_the_oracle_iteration_by_iteration(m, d, k, loo
         assert np.allclose(ha, ra, rtol=5e-3, atol=1e-9)
     else:
         assert np.allclose(ha[:3], ra[:3], rtol=5e-2)
+
+
+def test_dual_step_kernel_routes_collapsing_layers_like_two_launches():
+    """Batched scalar layers of which some collapse in mid-loop (tau above the mean absolute deviation of their
+    weights): the kernel that steps fp32 and fp64 layers side by side must route every layer exactly as two ordered
+    launches do -- bitwise equal centroids over many repeats, every arrival counter back at rest, and the oracle's
+    centroids per layer (which the collapsing layers only reach through the fp64 step)."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    shapes = [(16, 512, 3, 3), (64, 64, 3, 3), (24, 512, 3, 3), (32, 256, 3, 3), (8, 512, 3, 3), (40, 128, 3, 3),
+              (12, 512, 3, 3)]
+    wl = WL.config3(shapes=shapes, iters=40)
+    offs = [int(x) for x in wl.layer_offsets]
+    W, C0 = torch.from_numpy(wl.W).cuda(), torch.from_numpy(wl.C0).cuda()
+    ref = None
+    for method in (2, 1):
+        ctx = B.Context()
+        ctx.set_forward_loop(method)
+        for rep in range(1 if method == 2 else 25):
+            C = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter, layer_offsets=offs, want_Wq=False).C
+            torch.cuda.synchronize()
+            assert ctx.busy_tickets() == 0
+            assert all(i.status == 0 and i.fwd_iters == wl.max_iter for i in ctx.info())
+            if ref is None:
+                ref = C.cpu().numpy()
+            else:
+                assert np.array_equal(C.cpu().numpy(), ref), f"repeat {rep}"
+    # tolerance mode: layers leave the loop at different iterations
+    its = []
+    for method in (2, 1):
+        ctx = B.Context()
+        ctx.set_forward_loop(method)
+        Ct = ctx.forward(W, C0, wl.tau, 1e-5, 300, layer_offsets=offs, want_Wq=False).C.cpu().numpy()
+        assert ctx.busy_tickets() == 0
+        its.append(([i.fwd_iters for i in ctx.info()], Ct))
+    assert its[0][0] == its[1][0] and np.array_equal(its[0][1], its[1][1])
+    k = wl.k
+    for l, lw in enumerate(WL.split_layers(wl)):
+        r = oracle_run(lw, want_dW=False)
+        assert_close(ref[l * k:(l + 1) * k], r["C"], TOL_C, f"layer {l} C")

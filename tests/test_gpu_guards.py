@@ -4,8 +4,6 @@ Guard words: every output and the workspace sit inside a larger buffer filled wi
 sentinels before and after each of them must be intact.  Timeout path: the single-launch forward loop is told (host-side
 fault injection) to wait for an arrival that never comes; its bounded waits must run out, the status must say so and
 the context must stay usable."""
-import os
-
 import numpy as np
 import pytest
 
@@ -76,8 +74,7 @@ def test_barrier_timeout_is_reported_and_the_context_survives():
     ctx = B.Context()
     good = ctx.forward(W, C0, wl.tau, 0.0, 6).C.cpu().numpy()
     assert ctx.info()[0].status == 0
-    os.environ["IDKM_TEST_MISSING_ARRIVALS"] = "1"
-    os.environ["IDKM_TEST_SPIN_LIMIT"] = "2000000"          # about a millisecond
+    ctx.set_test_hooks(missing_arrivals=1, spin_limit_ticks=2000000)      # about a millisecond per wait
     try:
         ctx.forward(W, C0, wl.tau, 0.0, 6)
         torch.cuda.synchronize()
@@ -85,8 +82,7 @@ def test_barrier_timeout_is_reported_and_the_context_survives():
         assert info.status == B.ERR_TIMEOUT and info.fwd_iters == 0
         assert "wait" in B.status_string(B.ERR_TIMEOUT)
     finally:
-        del os.environ["IDKM_TEST_MISSING_ARRIVALS"]
-        del os.environ["IDKM_TEST_SPIN_LIMIT"]
+        ctx.set_test_hooks(0, 0)
     again = ctx.forward(W, C0, wl.tau, 0.0, 6).C.cpu().numpy()
     assert ctx.info()[0].status == 0 and ctx.info()[0].fwd_iters == 6
     assert np.array_equal(again, good)

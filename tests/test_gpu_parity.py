@@ -17,9 +17,11 @@ pytestmark = pytest.mark.gpu
 TOL_GRAD_KINK = 3e-2
 
 
-def check_workload(wl, modes=("implicit", "jfb"), alpha=1.0, want_A=False):
+def check_workload(wl, modes=("implicit", "jfb"), alpha=1.0, want_A=False, tag=None):
+    """`tag`: name under which the achieved errors go to the parity table (the configuration tests pass one)."""
     ctx = None
     for mode in modes:
+        rec = None if tag is None else f"{tag} [{mode}]"
         ref = oracle_run(wl, mode=mode, alpha=alpha, want_A=want_A)
         out = gpu_run(wl, mode=mode, alpha=alpha, want_A=want_A, ctx=ctx)
         ctx = out["ctx"]
@@ -27,11 +29,11 @@ def check_workload(wl, modes=("implicit", "jfb"), alpha=1.0, want_A=False):
         assert info.status == 0, info
         assert info.fwd_iters == wl.max_iter
         assert info.adj_iters == (wl.adj_max_iter if mode == "implicit" else 0)
-        assert_close(out["C"], ref["C"], TOL_C, f"{wl.name} C")
-        assert_close(out["Wq"], ref["Wq"], TOL_C, f"{wl.name} Wq")
+        assert_close(out["C"], ref["C"], TOL_C, f"{wl.name} C", record=rec)
+        assert_close(out["Wq"], ref["Wq"], TOL_C, f"{wl.name} Wq", record=rec)
         nx = kink_crossings(wl.W, out["C"], ref["C"])
-        assert_grad_close(out["dC"], ref["dC"], f"{wl.name} dC[{mode}]", nx, TOL_GRAD, TOL_GRAD_KINK)
-        assert_grad_close(out["dW"], ref["dW"], f"{wl.name} dW[{mode}]", nx, TOL_GRAD, TOL_GRAD_KINK)
+        assert_grad_close(out["dC"], ref["dC"], f"{wl.name} dC[{mode}] chained", nx, TOL_GRAD, TOL_GRAD_KINK, record=rec)
+        assert_grad_close(out["dW"], ref["dW"], f"{wl.name} dW[{mode}] chained", nx, TOL_GRAD, TOL_GRAD_KINK, record=rec)
         if want_A:
             assert np.abs(out["A"] - ref["A"]).max() <= 2e-6, "A"
             np.testing.assert_allclose(out["A"].sum(1), 1.0, atol=2e-6)
@@ -40,9 +42,9 @@ def check_workload(wl, modes=("implicit", "jfb"), alpha=1.0, want_A=False):
         refc = oracle_backward_at(wc, wc.C0, mode=mode, alpha=alpha)
         outc = gpu_run(wc, mode=mode, alpha=alpha, ctx=ctx)
         assert np.array_equal(outc["C"], wc.C0)
-        assert_close(outc["Wq"], refc["Wq"], TOL_C, f"{wl.name} Wq at common C")
-        assert_close(outc["dC"], refc["dC"], TOL_GRAD, f"{wl.name} dC[{mode}] at common C")
-        assert_close(outc["dW"], refc["dW"], TOL_GRAD, f"{wl.name} dW[{mode}] at common C")
+        assert_close(outc["Wq"], refc["Wq"], TOL_C, f"{wl.name} Wq at common C", record=rec)
+        assert_close(outc["dC"], refc["dC"], TOL_GRAD, f"{wl.name} dC[{mode}] at common C", record=rec)
+        assert_close(outc["dW"], refc["dW"], TOL_GRAD, f"{wl.name} dW[{mode}] at common C", record=rec)
 
 
 # sizes span one tile, several tiles and a ragged tail for every kernel layout (k picks the layout)
@@ -63,18 +65,18 @@ def test_small_cases_fixed_iterations(m, d, k):
 
 
 def test_config1():
-    check_workload(WL.config1())
+    check_workload(WL.config1(), tag="cfg1")
 
 
 def test_config1_paper_alpha():
     # the paper's averaged iteration, alpha = 0.25
-    check_workload(WL.config1(), modes=("implicit",), alpha=0.25)
+    check_workload(WL.config1(), modes=("implicit",), alpha=0.25, tag="cfg1 alpha=0.25")
 
 
 def test_config2_fixed_count():
     wl = WL.config2()
     wl.max_iter, wl.adj_max_iter = 60, 60
-    check_workload(wl)
+    check_workload(wl, tag="cfg2 60+60 fixed")
 
 
 def test_config2_tolerance_mode():
@@ -96,7 +98,15 @@ def test_config2_tolerance_mode():
     from oracle import idkm_ref as R
     Cn, _, _ = R.step(wl.W.astype(np.float64), out["C"].astype(np.float64), wl.tau)
     assert np.linalg.norm(Cn - out["C"]) / np.linalg.norm(Cn) < 2 * wl.tol
-    assert rel_err(out["dW"], ref["dW"])[0] < 1e-3
+    # The two runs stop where their own residual passes the tolerance, so their centroids differ by up to the
+    # tolerance and (d = 1) weights may lie between them; the backward is therefore held to the gradient tolerance
+    # at common centroids, with the adjoint run to the same tolerance on both sides.
+    wc = at_centroids(wl, ref["C"])
+    refc = oracle_run(wc, fixed=False)
+    outc = gpu_run(wc, fixed=False, ctx=out["ctx"])
+    assert abs(outc["info"][0].adj_iters - refc["adj_iters"]) <= 2
+    assert_close(outc["dC"], refc["dC"], TOL_GRAD, "cfg2 dC, tolerance mode, at common C", record="cfg2 tol 1e-6")
+    assert_close(outc["dW"], refc["dW"], TOL_GRAD, "cfg2 dW, tolerance mode, at common C", record="cfg2 tol 1e-6")
 
 
 def test_config3_batched_full():
@@ -112,29 +122,31 @@ def test_config3_batched_full():
         refs.append(ref)
         info = gpu["info"][l]
         assert info.status == 0 and info.fwd_iters == wl.max_iter and info.adj_iters == wl.adj_max_iter
-        assert_close(gpu["C"][l * k:(l + 1) * k], ref["C"], TOL_C, f"layer {l} C")
-        assert_close(gpu["Wq"][a:b], ref["Wq"], TOL_C, f"layer {l} Wq")
+        rec = f"cfg3 layer {l} (m = {b - a})"
+        assert_close(gpu["C"][l * k:(l + 1) * k], ref["C"], TOL_C, f"layer {l} C", record=rec)
+        assert_close(gpu["Wq"][a:b], ref["Wq"], TOL_C, f"layer {l} Wq", record=rec)
         nx = kink_crossings(lw.W, gpu["C"][l * k:(l + 1) * k], ref["C"])
         assert_grad_close(gpu["dC"][l * k:(l + 1) * k], ref["dC"], f"layer {l} dC", nx, TOL_GRAD, TOL_GRAD_KINK)
         assert_grad_close(gpu["dW"][a:b], ref["dW"], f"layer {l} dW", nx, TOL_GRAD, TOL_GRAD_KINK)
         refj = oracle_run(lw, mode="jfb")
         assert_grad_close(gpu_j["dC"][l * k:(l + 1) * k], refj["dC"], f"layer {l} dC jfb", nx, TOL_GRAD, TOL_GRAD_KINK)
         assert_grad_close(gpu_j["dW"][a:b], refj["dW"], f"layer {l} dW jfb", nx, TOL_GRAD, TOL_GRAD_KINK)
-    # the whole output tensors of the batched call, in the spec norm
-    assert_close(gpu["C"], np.concatenate([r["C"] for r in refs]), TOL_C, "C, all layers")
-    assert_close(gpu["Wq"], np.concatenate([r["Wq"] for r in refs]), TOL_C, "Wq, all layers")
+    # the whole output tensors of the batched call, in the stated norm
+    assert_close(gpu["C"], np.concatenate([r["C"] for r in refs]), TOL_C, "C, all layers", record="cfg3 all layers")
+    assert_close(gpu["Wq"], np.concatenate([r["Wq"] for r in refs]), TOL_C, "Wq, all layers", record="cfg3 all layers")
     # backward proper at common centroids, all layers in one batched call
     wc = at_centroids(wl, np.concatenate([r["C"] for r in refs]))
     gc = gpu_run(wc, mode="implicit", ctx=gpu["ctx"])
     gcj = gpu_run(wc, mode="jfb", ctx=gpu["ctx"])
     for l, lw in enumerate(WL.split_layers(wc)):
         a, b = int(wl.layer_offsets[l]), int(wl.layer_offsets[l + 1])
+        rec = f"cfg3 layer {l} (m = {b - a})"
         rc = oracle_backward_at(lw, lw.C0, mode="implicit")
-        assert_close(gc["dC"][l * k:(l + 1) * k], rc["dC"], TOL_GRAD, f"layer {l} dC at common C")
-        assert_close(gc["dW"][a:b], rc["dW"], TOL_GRAD, f"layer {l} dW at common C")
+        assert_close(gc["dC"][l * k:(l + 1) * k], rc["dC"], TOL_GRAD, f"layer {l} dC at common C", record=rec)
+        assert_close(gc["dW"][a:b], rc["dW"], TOL_GRAD, f"layer {l} dW at common C", record=rec)
         rj = oracle_backward_at(lw, lw.C0, mode="jfb")
-        assert_close(gcj["dC"][l * k:(l + 1) * k], rj["dC"], TOL_GRAD, f"layer {l} dC jfb at common C")
-        assert_close(gcj["dW"][a:b], rj["dW"], TOL_GRAD, f"layer {l} dW jfb at common C")
+        assert_close(gcj["dC"][l * k:(l + 1) * k], rj["dC"], TOL_GRAD, f"layer {l} dC jfb at common C", record=rec)
+        assert_close(gcj["dW"][a:b], rj["dW"], TOL_GRAD, f"layer {l} dW jfb at common C", record=rec)
 
 
 def test_batched_small_layers():
@@ -191,7 +203,7 @@ def test_batched_layers_with_row_cached_adjoint():
 
 def test_config4_reduced_m_full_k():
     wl = WL.config4(m=1 << 15, iters=20)
-    check_workload(wl)
+    check_workload(wl, tag="cfg4 reduced m = 2^15, 20+20")
 
 
 def test_run_to_run_bitwise_determinism():
@@ -256,13 +268,14 @@ def test_config4_full_size_against_stored_oracle_state():
     info = out["info"][0]
     assert info.status == 0 and info.fwd_iters == 50 and info.adj_iters == 50
     assert abs(info.fwd_residual - gold["fwd_residual"]) < 1e-3 * gold["fwd_residual"]
-    assert_close(out["C"], st["C"], TOL_C, "C")
+    rec = "cfg4 full size, 50+50"
+    assert_close(out["C"], st["C"], TOL_C, "C", record=rec)
     Wq_ref = R.final(Ws, st["C"], wl.tau)[0]
-    assert_close(out["Wq"][rows], Wq_ref, TOL_C, "Wq (sampled rows)")
-    # the adjoint after 50 not-yet-converged iterations at a contraction rate near 0.99 amplifies the 1e-6
-    # difference of the centroids; held to 1e-3 here and to the gradient tolerance at common centroids below
-    assert_close(out["dC"], st["u"], 1e-3, "dC chained")
-    assert_close(out["dW"][rows], R.scatter(Ws, Gs, st["C"], wl.tau, st["S"], st["F"], st["u"]), 1e-3, "dW chained")
+    assert_close(out["Wq"][rows], Wq_ref, TOL_C, "Wq (sampled rows)", record=rec)
+    # chained: the GPU's backward at the GPU's own centroids against the oracle's at the oracle's (d = 4: smooth)
+    assert_close(out["dC"], st["u"], TOL_GRAD, "dC chained", record=rec)
+    assert_close(out["dW"][rows], R.scatter(Ws, Gs, st["C"], wl.tau, st["S"], st["F"], st["u"]), TOL_GRAD,
+                 "dW chained (sampled rows)", record=rec)
 
     # backward proper at common centroids: C0 := fp32(oracle C_T), loop switched off
     sc = {key: np.array(v) for key, v in gold["at_fp32_C_T"].items() if isinstance(v, list)}
@@ -270,10 +283,10 @@ def test_config4_full_size_against_stored_oracle_state():
     assert np.array_equal(wc.C0.astype(np.float64), sc["C"])
     for mode, uref in (("implicit", sc["u"]), ("jfb", sc["g"])):
         oc = gpu_run(wc, mode=mode, ctx=out["ctx"])
-        assert_close(oc["dC"], uref, TOL_GRAD, f"dC {mode} at common C")
-        assert_close(oc["Wq"][rows], R.final(Ws, sc["C"], wl.tau)[0], TOL_C, "Wq at common C")
+        assert_close(oc["dC"], uref, TOL_GRAD, f"dC {mode} at common C", record=rec)
+        assert_close(oc["Wq"][rows], R.final(Ws, sc["C"], wl.tau)[0], TOL_C, "Wq at common C", record=rec)
         assert_close(oc["dW"][rows], R.scatter(Ws, Gs, sc["C"], wl.tau, sc["S"], sc["F"], uref), TOL_GRAD,
-                     f"dW {mode} at common C (sampled rows)")
+                     f"dW {mode} at common C (sampled rows)", record=rec)
     # invariants that hold at any size: rows of Wq lie in the bounding box of C; sum_j S_j = m
     assert np.all(out["Wq"] >= out["C"].min(0) - 1e-6) and np.all(out["Wq"] <= out["C"].max(0) + 1e-6)
     np.testing.assert_allclose(st["S"].sum(), wl.m, rtol=1e-12)
@@ -300,16 +313,17 @@ def test_sweep_point_fixed_iterations(m, d, b, tau):
     ref = oracle_run(wl, mode="implicit")
     out = gpu_run(wl, mode="implicit")
     assert out["info"][0].status == 0
-    assert_close(out["C"], ref["C"], TOL_C, "C")
-    assert_close(out["Wq"], ref["Wq"], TOL_C, "Wq")
+    rec = f"cfg5 m=2^{m.bit_length() - 1} d={d} k={1 << b} tau={tau}"
+    assert_close(out["C"], ref["C"], TOL_C, "C", record=rec)
+    assert_close(out["Wq"], ref["Wq"], TOL_C, "Wq", record=rec)
     nx = kink_crossings(wl.W, out["C"], ref["C"])
-    assert_grad_close(out["dC"], ref["dC"], "dC", nx, TOL_GRAD, TOL_GRAD_KINK)
-    assert_grad_close(out["dW"], ref["dW"], "dW", nx, TOL_GRAD, TOL_GRAD_KINK)
+    assert_grad_close(out["dC"], ref["dC"], "dC chained", nx, TOL_GRAD, TOL_GRAD_KINK, record=rec)
+    assert_grad_close(out["dW"], ref["dW"], "dW chained", nx, TOL_GRAD, TOL_GRAD_KINK, record=rec)
     # invariants that hold at any size
     assert np.all(out["Wq"] >= out["C"].min(0) - 1e-6) and np.all(out["Wq"] <= out["C"].max(0) + 1e-6)
     if nx:
         wc = at_centroids(wl, ref["C"])
         refc = oracle_backward_at(wc, wc.C0, mode="implicit")
         outc = gpu_run(wc, mode="implicit", ctx=out["ctx"])
-        assert_close(outc["dC"], refc["dC"], TOL_GRAD, "dC at common C")
-        assert_close(outc["dW"], refc["dW"], TOL_GRAD, "dW at common C")
+        assert_close(outc["dC"], refc["dC"], TOL_GRAD, "dC at common C", record=rec)
+        assert_close(outc["dW"], refc["dW"], TOL_GRAD, "dW at common C", record=rec)

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 ORACLE = os.path.join(ROOT, "oracle")
 
 MUTATIONS = [
-    ("squared distance in the softmax", "    D[j] = sqrt(s);", "    D[j] = s;"),
+    ("squared distance in the softmax", "    D[j] = g_squared ? s : sqrt(s);", "    D[j] = s;"),
     ("temperature dropped from the softmax", "A[j] = exp(-(D[j] - dmin) / tau);", "A[j] = exp(-(D[j] - dmin));"),
     ("M-step not normalised by the column sum", "C_plus[j * d + a] = N[j * d + a] / S[j];",
      "C_plus[j * d + a] = N[j * d + a] / (double)m;"),
@@ -35,6 +35,18 @@ MUTATIONS = [
      "for (int j = 0; j < k; ++j) s += A[k - 1 - j] * C[j * d + a];"),
 ]
 
+# the same for the squared-distance variant (the battery then runs with the variant switched on)
+MUTATIONS_SQUARED = [
+    ("variant ignores the switch in the distance", "    D[j] = g_squared ? s : sqrt(s);", "    D[j] = sqrt(s);"),
+    ("factor 2 of the squared distance's gradient dropped", "n[a] = 2.0 * (w[a] - cj[a]);", "n[a] = (w[a] - cj[a]);"),
+    ("squared distance's gradient normalised like the unit vector", "n[a] = 2.0 * (w[a] - cj[a]);",
+     "n[a] = (Dj > 0.0) ? (w[a] - cj[a]) / sqrt(Dj) : 0.0;"),
+    ("sign of the squared distance's gradient", "n[a] = 2.0 * (w[a] - cj[a]);", "n[a] = 2.0 * (cj[a] - w[a]);"),
+    ("mean subtraction dropped in the adjoint", "double e = A[j] * (p[j] - s);", "double e = A[j] * p[j];"),
+    ("1/tau dropped from the codebook gradient", "pg[j * d + a] += A[j] * Gi[a] + (e / tau) * n[a];",
+     "pg[j * d + a] += A[j] * Gi[a] + e * n[a];"),
+]
+
 
 def _load_mutant(tmp_path, old, new):
     src = open(os.path.join(ORACLE, "idkm_ref.c")).read()
@@ -52,10 +64,19 @@ def _load_mutant(tmp_path, old, new):
 def test_unmutated_oracle_passes_the_battery():
     from oracle import idkm_ref as R
     assert run_battery(R) == []
+    assert run_battery(R, squared=True) == []
+    assert R.get_squared() is False          # the battery leaves the oracle in the published setting
 
 
 @pytest.mark.parametrize("name,old,new", MUTATIONS, ids=[m[0] for m in MUTATIONS])
 def test_battery_catches_planted_mistake(tmp_path, name, old, new):
     mutant = _load_mutant(tmp_path, old, new)
     failed = run_battery(mutant)
+    assert failed, f"no pin noticed: {name}"
+
+
+@pytest.mark.parametrize("name,old,new", MUTATIONS_SQUARED, ids=[m[0] for m in MUTATIONS_SQUARED])
+def test_battery_catches_planted_mistake_in_the_squared_variant(tmp_path, name, old, new):
+    mutant = _load_mutant(tmp_path, old, new)
+    failed = run_battery(mutant, squared=True)
     assert failed, f"no pin noticed: {name}"

@@ -18,7 +18,8 @@ def _regular_one_step(ctx, W, C0, tau):
     return ctx.forward(W, C0, tau, 0.0, 1, want_Wq=False).C
 
 
-@pytest.mark.parametrize("m,d,k,tau", [(50001, 1, 4, 0.01), (30011, 4, 64, 0.012), (20000, 2, 256, 0.01)])
+@pytest.mark.parametrize("m,d,k,tau", [(50001, 1, 4, 0.01), (30011, 4, 64, 0.012), (20000, 2, 256, 0.01),
+                                       (30000, 4, 256, 0.012), (30000, 1, 256, 0.01)])
 def test_noalloc_step_matches_regular_forward_twice(m, d, k, tau):
     import torch
     from paper_2312_07759_b200 import binding as B
@@ -52,6 +53,42 @@ def test_noalloc_collapsed_start_takes_the_fp64_step():
     ref = _regular_one_step(B.Context(), W, torch.from_numpy(C0).cuda(), wl.tau)
     torch.cuda.synchronize()
     assert_close(out.cpu().numpy(), ref.cpu().numpy(), TOL_C, "collapsed start")
+
+
+def test_noalloc_every_supported_codebook_fits_the_builtin_scratch():
+    """The size check passes for every (d, codebook layout) on a layer large enough to fill the grid, the largest
+    codebook included; the result still matches the regular entry point."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    ctx = B.Context()
+    for d in (1, 2, 4):
+        for k in (2, 4, 8, 16, 32, 64, 128, 256):
+            m = 400000
+            wl = WL.single_layer(m, d, k, 0.012, std=0.03, seed=d * 1000 + k, init="rows")
+            W, C0 = torch.from_numpy(wl.W).cuda(), torch.from_numpy(wl.C0).cuda()
+            out = torch.empty_like(C0)
+            rc = B.lib.idkm_step_noalloc(W.data_ptr(), m, d, C0.data_ptr(), k, wl.tau, out.data_ptr(), None)
+            assert rc == B.OK, (d, k, rc)
+            ref = _regular_one_step(ctx, W, C0, wl.tau)
+            torch.cuda.synchronize()
+            assert B.step_noalloc_status() == B.OK
+            assert_close(out.cpu().numpy(), ref.cpu().numpy(), TOL_C, f"d={d} k={k}")
+
+
+def test_noalloc_status_reports_a_nan_in_the_weights():
+    """The step has no context to report through: a NaN in W must show in idkm_step_noalloc_status, and a clean call
+    afterwards must read OK again."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(30000, 1, 4, 0.01, std=0.03, seed=2)
+    Wbad = wl.W.copy()
+    Wbad[1234, 0] = np.nan
+    C0 = torch.from_numpy(wl.C0).cuda()
+    B.step_noalloc(torch.from_numpy(Wbad).cuda(), C0, wl.tau)
+    assert B.step_noalloc_status() == B.ERR_NONFINITE
+    B.step_noalloc(torch.from_numpy(wl.W).cuda(), C0, wl.tau)
+    assert B.step_noalloc_status() == B.OK
+    assert B.lib.idkm_step_noalloc_status(None, None) == B.ERR_NULL
 
 
 def test_noalloc_argument_errors():
