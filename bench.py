@@ -144,6 +144,24 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}, "fallback"
 
 
+def stored_traffic(workload_name):
+    """DRAM bytes per launch of the loop kernels from the stored ncu capture (profiles/traffic_cfg4.json): a map
+    "<pass>:<centroids per lane>x<lanes per weight>" -> bytes, empty when the file is for another workload or was
+    written for another version of the kernel source."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "traffic_cfg4.json")
+    src = os.path.join(ROOT, "paper_2312_07759_b200", "csrc", "idkm_kernels.cuh")
+    if workload_name is None or not os.path.exists(path) or not os.path.exists(src):
+        return {}
+    with open(path) as f:
+        t = json.load(f)
+    with open(src, "rb") as f:
+        sha = hashlib.sha256(f.read()).hexdigest()
+    if t.get("workload") != workload_name or t.get("kernel_source_sha256") != sha:
+        return {}
+    return {key: v["dram_bytes_read"] + v["dram_bytes_write"] for key, v in t.get("kernels", {}).items()}
+
+
 def time_oracle_sample(wl, rows: int, it_f: int, it_a: int):
     """Times the float64 oracle on the first `rows` rows of the workload: it_f forward iterations and it_a
     adjoint iterations (plus the final pass and the codebook gradient they need).  Returns
@@ -284,74 +302,91 @@ def main():
     step_kernel_ms = ph["steps"] / max(T_f, 1)
     adj_kernel_ms = ph["adjoint"] / max(T_a, 1)
 
-    # ---- roofline of the dominant kernel (the fused forward step) ---------------------------------------------
-    fp32_ops, sfu_ops = pair_ops(d)
+    # ---- rooflines of the two loop kernels; `roofline` is the one with the larger share of the step -----------------
     pairs = float(m) * k
     peaks, which = measured_peaks()
-    t_hbm = (4.0 * d * m) / (peaks["hbm_gbs"] * 1e9)
-    t_fp32 = pairs * fp32_ops / (SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6)
-    t_sfu = pairs * sfu_ops / (SM_COUNT * SFU_LANES_PER_SM * SM_MAX_MHZ * 1e6)
-    if t_hbm >= max(t_fp32, t_sfu):
-        roof = {"bound": "hbm", "achieved": 4.0 * d * m / (step_kernel_ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                "unit": "GB/s", "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({which})"}
-    elif t_fp32 >= t_sfu:
-        roof = {"bound": "alu", "achieved": pairs * fp32_ops / (step_kernel_ms * 1e-3) / 1e12,
-                "peak": SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12, "unit": "Tinst-lanes/s (fp32 pipe)",
-                "peak_source": "148 SMs x 128 fp32 lanes/clk x 1965 MHz"}
-    else:
-        roof = {"bound": "alu", "achieved": pairs * sfu_ops / (step_kernel_ms * 1e-3) / 1e12,
-                "peak": SM_COUNT * SFU_LANES_PER_SM * SM_MAX_MHZ * 1e6 / 1e12, "unit": "Tinst-lanes/s (sfu pipe)",
-                "peak_source": "148 SMs x 16 sfu lanes/clk x 1965 MHz"}
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["kernel"] = "idkm_pass<STEP> (fused forward step)"
-    roof["kernel_ms"] = step_kernel_ms
-    # dram__bytes_read.sum + dram__bytes_write.sum of one launch, from profiles/step_kernel_cfg4.txt (ncu flushes the
-    # caches before the launch, so this is the cold-L2 figure); only known for the profiled workload
-    roof["traffic"] = 67.21e6 + 0.59e6 if wl.name.startswith("cfg4_vq_m4194304") and args.iters == 0 else None
-    roof["roofline_ms"] = max(t_hbm, t_fp32, t_sfu) * 1e3
-    # the same two pipes measured now by the library's register-only micro-benchmarks (at the clock of an otherwise
-    # idle GPU): the nominal peak above is the contract figure, this one shows how much of it the hardware delivers
-    fp32_rate, sfu_rate = B.measure_pipe_rates()
-    roof["pipes_measured"] = {"fp32_lane_ops_per_s": fp32_rate, "sfu_lane_ops_per_s": sfu_rate,
-                              "fp32_lanes_per_clk_per_sm_at_max_clock": fp32_rate / (SM_COUNT * SM_MAX_MHZ * 1e6),
-                              "sfu_lanes_per_clk_per_sm_at_max_clock": sfu_rate / (SM_COUNT * SM_MAX_MHZ * 1e6)}
-    roof["frac_of_measured_pipes"] = max(t_hbm, pairs * fp32_ops / fp32_rate, pairs * sfu_ops / sfu_rate) \
-        / (step_kernel_ms * 1e-3)
-    # the adjoint step takes the larger share of the step's time: the same arithmetic for it
-    a_fp32, a_sfu = adjoint_pair_ops(d)
-    ta_fp32 = pairs * a_fp32 / (SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6)
-    ta_sfu = pairs * a_sfu / (SM_COUNT * SFU_LANES_PER_SM * SM_MAX_MHZ * 1e6)
-    ta = max(t_hbm, ta_fp32, ta_sfu)
-    roof_adj = None
-    if T_a > 0 and adj_kernel_ms > 0 and k * d > 8:     # smaller codebooks take the explicit-Jacobian path
-        roof_adj = {"kernel": "idkm_pass<ADJ> (fused adjoint step)", "kernel_ms": adj_kernel_ms, "roofline_ms": ta * 1e3,
-                    "bound": "hbm" if ta == t_hbm else "alu", "frac": ta / (adj_kernel_ms * 1e-3),
-                    "fp32_ops_per_pair": a_fp32, "sfu_ops_per_pair": a_sfu}
+    fp32_rate, sfu_rate = B.measure_pipe_rates()      # register-only micro-benchmarks of the two pipes, measured now
+    path = B.describe_path(d, k, T_a, 0)
+    traffic_table = stored_traffic(wl.name if args.iters == 0 else None)
 
-    # ---- end to end through the host-buffer entry point ----------------------------------------------------------
+    def kernel_roofline(label, layout, kernel_ms, ops, share):
+        fp32_ops, sfu_ops = ops
+        t_hbm = (4.0 * d * m) / (peaks["hbm_gbs"] * 1e9)
+        fp32_peak = SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6
+        sfu_peak = SM_COUNT * SFU_LANES_PER_SM * SM_MAX_MHZ * 1e6
+        t_fp32, t_sfu = pairs * fp32_ops / fp32_peak, pairs * sfu_ops / sfu_peak
+        sec = kernel_ms * 1e-3
+        if t_hbm >= max(t_fp32, t_sfu):
+            r = {"bound": "hbm", "achieved": 4.0 * d * m / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                 "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({which})"}
+        elif t_fp32 >= t_sfu:
+            r = {"bound": "alu", "achieved": pairs * fp32_ops / sec / 1e12, "peak": fp32_peak / 1e12,
+                 "unit": "Tinst-lanes/s (fp32 pipe)", "peak_source": "148 SMs x 128 fp32 lanes/clk x 1965 MHz"}
+        else:
+            r = {"bound": "alu", "achieved": pairs * sfu_ops / sec / 1e12, "peak": sfu_peak / 1e12,
+                 "unit": "Tinst-lanes/s (sfu pipe)", "peak_source": "148 SMs x 16 sfu lanes/clk x 1965 MHz"}
+        r["frac"] = r["achieved"] / r["peak"]
+        r["kernel"] = f"{label}, layout {layout[0]} centroids/lane x {layout[1]} lanes/weight"
+        r["kernel_ms"] = kernel_ms
+        r["share_of_step"] = share
+        r["roofline_ms"] = max(t_hbm, t_fp32, t_sfu) * 1e3
+        r["fp32_ops_per_pair"], r["sfu_ops_per_pair"] = fp32_ops, sfu_ops
+        # dram__bytes_read.sum + dram__bytes_write.sum of one launch from the stored ncu capture of this kernel (ncu
+        # flushes the caches before the launch, so this is the cold-L2 figure); null when none is stored for this
+        # workload and layout, or when the kernel source has changed since the capture
+        r["traffic"] = traffic_table.get(f"{label.split(' ')[0]}:{layout[0]}x{layout[1]}")
+        r["frac_of_measured_pipes"] = max(t_hbm, pairs * fp32_ops / fp32_rate, pairs * sfu_ops / sfu_rate) / sec
+        return r
+
+    step_total = float(np.mean(step_ms))
+    roof_step = kernel_roofline("idkm_pass<STEP> (fused forward step)", path["step_layout"], step_kernel_ms, pair_ops(d),
+                                ph["steps"] / step_total) if T_f > 0 and step_kernel_ms > 0 else None
+    roof_adj = None
+    if T_a > 0 and adj_kernel_ms > 0 and path["adjoint_route"] == "fused passes":
+        roof_adj = kernel_roofline("idkm_pass<ADJ> (fused adjoint step)", path["adjoint_layout"], adj_kernel_ms,
+                                   adjoint_pair_ops(d), ph["adjoint"] / step_total)
+    ranked = sorted([r for r in (roof_step, roof_adj) if r is not None], key=lambda r: -r["share_of_step"])
+    roof = ranked[0] if ranked else None
+    roof_second = ranked[1] if len(ranked) > 1 else None
+    if roof is not None:
+        roof["pipes_measured"] = {"fp32_lane_ops_per_s": fp32_rate, "sfu_lane_ops_per_s": sfu_rate,
+                                  "fp32_lanes_per_clk_per_sm_at_max_clock": fp32_rate / (SM_COUNT * SM_MAX_MHZ * 1e6),
+                                  "sfu_lanes_per_clk_per_sm_at_max_clock": sfu_rate / (SM_COUNT * SM_MAX_MHZ * 1e6)}
+        roof["adjoint_route"] = path["adjoint_route"]
+
+    # ---- end to end through the host-buffer entry point: the same work as the timed step ----------------------------
     e2e = None
     if not args.no_e2e:
         hW = torch.from_numpy(wl.W).pin_memory()
         hG = torch.from_numpy(wl.G).pin_memory()
         hC0 = torch.from_numpy(wl.C0).pin_memory()
         outs = {"C": torch.empty_like(hC0).pin_memory().numpy(), "Wq": torch.empty_like(hW).pin_memory().numpy(),
-                "dW": torch.empty_like(hW).pin_memory().numpy(), "dC": torch.empty_like(hC0).pin_memory().numpy()}
+                "dW": torch.empty_like(hW).pin_memory().numpy(), "dC": torch.empty_like(hC0).pin_memory().numpy(),
+                "dW_jfb": torch.empty_like(hW).pin_memory().numpy(), "dC_jfb": torch.empty_like(hC0).pin_memory().numpy()}
         hctx = B.Context()
         n_e2e = max(2, min(args.steps, 3))
-        hctx.quantize_host(hW.numpy(), hC0.numpy(), hG.numpy(), wl.tau, 0.0, T_f, B.IMPLICIT, 0.0, T_a, 1.0,
-                           layer_offsets=offs, out=outs)
+
+        def host_step():
+            # forward + Jacobian-free backward + implicit backward from one forward, as in step() above
+            return hctx.quantize_host(hW.numpy(), hC0.numpy(), hG.numpy(), wl.tau, 0.0, T_f, B.IMPLICIT, 0.0, T_a, 1.0,
+                                      layer_offsets=offs, out=outs, also_jfb=True)
+
+        host_step()
         barrier()
-        t0 = time.perf_counter()
+        e2e_ms = []
         for _ in range(n_e2e):
-            hctx.quantize_host(hW.numpy(), hC0.numpy(), hG.numpy(), wl.tau, 0.0, T_f, B.IMPLICIT, 0.0, T_a, 1.0,
-                               layer_offsets=offs, out=outs)
-        torch.cuda.synchronize()
-        e2e_s = (time.perf_counter() - t0) / n_e2e
-        e2e_s = max_over_ranks(e2e_s, dev)
+            flush.fill_(3)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            host_step()                      # returns after the last copy has landed
+            e2e_ms.append((time.perf_counter() - t0) * 1e3)
+        e2e_s = max_over_ranks(float(np.mean(e2e_ms)) * 1e-3, dev)
         e2e = {"value": job_value(m, T_f + T_a, world, e2e_s * 1e3), "unit": "weight-iterations/s",
                "h2d_bytes_per_step": int(hW.numel() * 4 + hG.numel() * 4 + hC0.numel() * 4),
-               "d2h_bytes_per_step": int(2 * hW.numel() * 4 + 2 * hC0.numel() * 4), "ms_per_step": e2e_s * 1e3,
-               "api": "idkm_quantize_host (forward + implicit backward, pinned host buffers)"}
+               "d2h_bytes_per_step": int(3 * hW.numel() * 4 + 3 * hC0.numel() * 4), "ms_per_step": e2e_s * 1e3,
+               "api": "idkm_quantize_host_ex (forward + Jacobian-free backward + implicit backward, pinned host "
+                      "buffers; the upload of dL/dWq overlaps the forward loop, the downloads of Wq and the "
+                      "Jacobian-free dL/dW overlap the backward)"}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -373,7 +408,7 @@ def main():
             "adjoint_wit_per_s": world * m * T_a / (ph["adjoint"] * 1e-3) if T_a else None,
             "step_ms": [round(x, 3) for x in step_ms],
             "step_phase_sum_ms": [round(sum(p.values()), 3) for p in phases], "phase_ms": ph, "step_kernel_ms": step_kernel_ms, "adjoint_kernel_ms": adj_kernel_ms,
-            "roofline": roof, "roofline_adjoint": roof_adj, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(n_launch), "clocks": clocks,
+            "roofline": roof, "roofline_second": roof_second, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(n_launch), "clocks": clocks,
             "info": {"status": [i.status for i in info][:4], "fwd_residual": info[0].fwd_residual,
                      "adj_residual": info[0].adj_residual},
         }

@@ -155,14 +155,29 @@ int idkm_get_history(idkm_ctx* ctx, int which, int layer, float* host_out, int c
  * Whole hot path on HOST buffers (Algorithm 2's per-layer work: cluster, quantise, differentiate):
  * copies W, C0 and dWq to the device, runs idkm_forward_batched and idkm_backward, and copies
  * C, Wq, dW, dC back; returns after everything has completed.  Device buffers are allocated on
- * first use, kept in the ctx and grown on demand (this is the only entry point that allocates
- * device memory).  Any of Wq_out, dW_out, dC_out may be NULL; info_out (n_layers entries) too.
+ * first use, kept in the ctx and grown on demand (with idkm_quantize_host_ex the only entry point that
+ * allocates device memory); the work runs on two streams of the ctx's own, so that the upload of dWq
+ * overlaps the forward loop and the download of C and Wq overlaps the backward (host buffers must be
+ * page-locked for the overlap to happen; pageable buffers work, serially).
+ * Any of Wq_out, dW_out, dC_out may be NULL; info_out (n_layers entries) too.
  * layer_offsets as in idkm_forward_batched (pass {0, m} and n_layers = 1 for one layer).
  */
 int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
                        const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
                        idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
                        float* Wq_out_host, float* dW_out_host, float* dC_out_host, idkm_info* info_out);
+
+/*
+ * The same with both gradients of Sections 4.2 and 4.3 from one forward: when mode is IDKM_IMPLICIT and
+ * dW_jfb_out_host or dC_jfb_out_host is given (HOST, shapes of dW_out / dC_out), the Jacobian-free backward
+ * (IDKM_JFB) runs as well, after the forward and before the implicit backward, and its results are copied there.
+ * With both NULL this is idkm_quantize_host.  info_out describes the implicit backward.
+ */
+int idkm_quantize_host_ex(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
+                          const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
+                          idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
+                          float* Wq_out_host, float* dW_out_host, float* dC_out_host, float* dW_jfb_out_host,
+                          float* dC_jfb_out_host, idkm_info* info_out);
 
 /*
  * Phase timing.  idkm_set_timing(ctx, 1) makes the following forward / backward calls record CUDA
@@ -286,6 +301,16 @@ int idkm_set_test_hooks(idkm_ctx* ctx, int missing_arrivals, int64_t spin_limit_
  * some blocks and never finished.  Returns IDKM_OK, IDKM_ERR_NULL, IDKM_ERR_ORDER (no forward yet) or IDKM_ERR_CUDA.
  */
 int idkm_count_busy_tickets(idkm_ctx* ctx, int* count_out);
+
+/*
+ * Which kernels the library picks for a problem shape (for benchmarks that attribute time to kernels).  Writes five
+ * ints to the HOST array out: [0], [1] centroids per lane and lanes per weight-vector of the fused forward step
+ * (Algorithm 1, steps 3-5); [2], [3] the same of the fused adjoint step (Section 4.2); [4] how an implicit backward
+ * of adj_max_iter steps with idkm_set_adjoint_method = adjoint_method runs the iteration: 0 one fused pass per step,
+ * 1 explicit k d x k d matrix held in registers (k d <= 8), 2 explicit matrix in tiles (k d <= 64, from 16 steps).
+ * Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_UNSUPPORTED.  Needs no device.
+ */
+int idkm_describe_path(int d, int k, int adj_max_iter, int adjoint_method, int* out);
 
 /* Number of kernels this ctx has launched since idkm_create (for accounting in benchmarks). */
 int64_t idkm_launch_count(const idkm_ctx* ctx);

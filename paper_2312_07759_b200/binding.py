@@ -55,6 +55,10 @@ lib.idkm_get_info.restype = C.c_int
 lib.idkm_quantize_host.argtypes = [_vp, _fp, _i64p, C.c_int, C.c_int, _fp, C.c_int, C.c_float, C.c_float, C.c_int,
                                    _fp, C.c_int, C.c_float, C.c_int, C.c_float, _fp, _fp, _fp, _fp, C.POINTER(Info)]
 lib.idkm_quantize_host.restype = C.c_int
+lib.idkm_quantize_host_ex.argtypes = [_vp, _fp, _i64p, C.c_int, C.c_int, _fp, C.c_int, C.c_float, C.c_float, C.c_int,
+                                      _fp, C.c_int, C.c_float, C.c_int, C.c_float, _fp, _fp, _fp, _fp, _fp, _fp,
+                                      C.POINTER(Info)]
+lib.idkm_quantize_host_ex.restype = C.c_int
 lib.idkm_set_timing.argtypes = [_vp, C.c_int]
 lib.idkm_set_timing.restype = C.c_int
 lib.idkm_get_phase_ms.argtypes = [_vp, C.POINTER(C.c_float)]
@@ -73,6 +77,8 @@ lib.idkm_get_history.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(C.c_float), C.
 lib.idkm_get_history.restype = C.c_int
 lib.idkm_set_forward_loop.argtypes = [_vp, C.c_int]
 lib.idkm_set_forward_loop.restype = C.c_int
+lib.idkm_describe_path.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int)]
+lib.idkm_describe_path.restype = C.c_int
 lib.idkm_launch_count.argtypes = [_vp]
 lib.idkm_launch_count.restype = C.c_int64
 lib.idkm_measure_pipe_rates.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_double), _vp]
@@ -155,6 +161,14 @@ def assign(W, Cm, want_codes: bool = True, want_Wq: bool = True, stream=None):
     _check(lib.idkm_assign(_ptr(W), m, d, _ptr(Cm), k, _ptr(codes) if codes is not None else None,
                            _ptr(Wq) if Wq is not None else None, _stream(stream)))
     return codes, Wq
+
+
+def describe_path(d: int, k: int, adj_max_iter: int = 0, adjoint_method: int = 0) -> dict:
+    """``idkm_describe_path``: the kernel layouts and the adjoint route the library picks for (d, k)."""
+    out = (C.c_int * 5)()
+    _check(lib.idkm_describe_path(int(d), int(k), int(adj_max_iter), int(adjoint_method), out))
+    return {"step_layout": (out[0], out[1]), "adjoint_layout": (out[2], out[3]),
+            "adjoint_route": ("fused passes", "explicit Jacobian in registers", "explicit Jacobian in tiles")[out[4]]}
 
 
 def measure_pipe_rates(stream=None):
@@ -246,10 +260,12 @@ class Context:
         return list(arr)
 
     def quantize_host(self, W, C0, G, tau, tol, max_iter, mode=IMPLICIT, adj_tol=0.0, adj_max_iter=30, alpha=1.0,
-                      layer_offsets=None, want_Wq=True, want_dW=True, out=None):
+                      layer_offsets=None, want_Wq=True, want_dW=True, out=None, also_jfb=False):
         """``idkm_quantize_host`` on HOST arrays (numpy float32, C-contiguous; pinned memory is the caller's choice).
 
-        ``out`` may carry preallocated host arrays {"C", "Wq", "dW", "dC"} to write into."""
+        ``out`` may carry preallocated host arrays {"C", "Wq", "dW", "dC", "dW_jfb", "dC_jfb"} to write into.  With
+        ``also_jfb`` (``idkm_quantize_host_ex``) the Jacobian-free gradients are computed from the same forward and
+        returned as two more arrays after the info list."""
         import numpy as np
         m, d = W.shape
         if layer_offsets is None:
@@ -264,6 +280,15 @@ class Context:
         offs = (C.c_int64 * (L + 1))(*[int(x) for x in layer_offsets])
         infos = (Info * L)()
         hp = lambda a: None if a is None else a.ctypes.data
+        if also_jfb:
+            dWj = out.get("dW_jfb") if out.get("dW_jfb") is not None else np.empty_like(W)
+            dCj = out.get("dC_jfb") if out.get("dC_jfb") is not None else np.empty_like(C0)
+            rc = lib.idkm_quantize_host_ex(self._h, hp(W), offs, L, d, hp(C0), k, float(tau), float(tol), int(max_iter),
+                                           hp(G), int(mode), float(adj_tol), int(adj_max_iter), float(alpha), hp(Cout),
+                                           hp(Wq), hp(dW), hp(dC), hp(dWj), hp(dCj), infos)
+            _check(rc)
+            self.n_layers = L
+            return Cout, Wq, dW, dC, list(infos), dWj, dCj
         rc = lib.idkm_quantize_host(self._h, hp(W), offs, L, d, hp(C0), k, float(tau), float(tol), int(max_iter), hp(G),
                                     int(mode), float(adj_tol), int(adj_max_iter), float(alpha), hp(Cout), hp(Wq), hp(dW),
                                     hp(dC), infos)

@@ -103,6 +103,9 @@ int pick_family(int mode, int d, int k) {
   // per SM is faster than 16 centroids per lane on half-warps (m = 2^22, k = 256: d = 1 0.46 against 0.54 ms, d = 2
   // 0.71 against 0.77 ms); for d = 4 the half-warp layout wins (0.90 against 0.95 ms)
   if (mode == STEP && k > 128 && d < 4) return N_FAMILY - 1;
+  // adjoint step with more than 128 centroids at d = 4: 16 centroids per lane on half-warps (m = 2^22, k = 256:
+  // 1.22 against 1.29 ms for 8 per lane on full warps)
+  if (mode == ADJ && k > 128 && d == 4) return N_FAMILY - 1;
   for (int f = 0; f < N_FAMILY; ++f) {
     const KernelEntry* e = kernel_entry(mode, d, f);
     if (e && e->launch && e->kpl * e->lpw >= k) return f;
@@ -225,9 +228,12 @@ struct idkm_ctx {
   long long row_off[MAX_LAYERS + 1];
   cudaStream_t stream;
   int occupancy[N_MODES][3][N_FAMILY];   // cached blocks/SM per kernel, 0 = not queried
-  // device buffers of the host-pointer entry point
+  // device buffers, streams and events of the host-pointer entry point
   void* hbuf;
   size_t hbuf_bytes;
+  bool host_streams_ok;
+  cudaStream_t hs_compute, hs_copy;
+  cudaEvent_t hev[4];
   // optional phase timing (CUDA events on the call's stream)
   bool timing;
   bool ev_ok;
@@ -519,6 +525,11 @@ int idkm_create(idkm_ctx** out) {
 void idkm_destroy(idkm_ctx* ctx) {
   if (!ctx) return;
   if (ctx->hbuf) cudaFree(ctx->hbuf);
+  if (ctx->host_streams_ok) {
+    for (int i = 0; i < 4; ++i) cudaEventDestroy(ctx->hev[i]);
+    cudaStreamDestroy(ctx->hs_compute);
+    cudaStreamDestroy(ctx->hs_copy);
+  }
   if (ctx->chunk_ev_ok) {
     cudaEventDestroy(ctx->chunk_ev[0]);
     cudaEventDestroy(ctx->chunk_ev[1]);
@@ -693,10 +704,11 @@ int idkm_get_info(idkm_ctx* ctx, idkm_info* info_out) {
   return IDKM_OK;
 }
 
-int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
-                       const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
-                       idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
-                       float* Wq_out_host, float* dW_out_host, float* dC_out_host, idkm_info* info_out) {
+int idkm_quantize_host_ex(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
+                          const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
+                          idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
+                          float* Wq_out_host, float* dW_out_host, float* dC_out_host, float* dW_jfb_out_host,
+                          float* dC_jfb_out_host, idkm_info* info_out) {
   if (!ctx || !W_host || !layer_offsets || !C0_host || !dWq_host || !C_out_host) return IDKM_ERR_NULL;
   if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K) return IDKM_ERR_UNSUPPORTED;
   if (n_layers < 1 || n_layers > IDKM_MAX_LAYERS || layer_offsets[0] != 0) return IDKM_ERR_SHAPE;
@@ -704,10 +716,11 @@ int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_
   if (m < 1) return IDKM_ERR_SHAPE;
   const size_t ws_bytes = idkm_workspace_bytes(m, d, k, n_layers);
   if (ws_bytes == 0) return IDKM_ERR_UNSUPPORTED;
+  const bool also_jfb = (dW_jfb_out_host != nullptr || dC_jfb_out_host != nullptr) && mode == IDKM_IMPLICIT;
   const size_t wbytes = align_up(sizeof(float) * (size_t)m * d, 256);
   const size_t cbytes = align_up(sizeof(float) * (size_t)n_layers * k * d, 256);
-  // W, G, Wq, dW | C0, C, dC | workspace
-  const size_t need = 4 * wbytes + 3 * cbytes + align_up(ws_bytes, 256);
+  // W, G, Wq, dW, dW (Jacobian-free) | C0, C, dC, dC (Jacobian-free) | workspace
+  const size_t need = 5 * wbytes + 4 * cbytes + align_up(ws_bytes, 256);
   if (need > ctx->hbuf_bytes) {
     if (ctx->hbuf) cudaFree(ctx->hbuf);
     ctx->hbuf = nullptr;
@@ -718,34 +731,78 @@ int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_
     }
     ctx->hbuf_bytes = need;
   }
+  // two streams of the ctx's own: the kernels run on one, the copies that can overlap them on the other
+  if (!ctx->host_streams_ok) {
+    if (cudaStreamCreateWithFlags(&ctx->hs_compute, cudaStreamNonBlocking) != cudaSuccess) return IDKM_ERR_CUDA;
+    if (cudaStreamCreateWithFlags(&ctx->hs_copy, cudaStreamNonBlocking) != cudaSuccess) {
+      cudaStreamDestroy(ctx->hs_compute);
+      return IDKM_ERR_CUDA;
+    }
+    for (int i = 0; i < 4; ++i)
+      if (cudaEventCreateWithFlags(&ctx->hev[i], cudaEventDisableTiming) != cudaSuccess) {
+        for (int q = 0; q < i; ++q) cudaEventDestroy(ctx->hev[q]);
+        cudaStreamDestroy(ctx->hs_compute);
+        cudaStreamDestroy(ctx->hs_copy);
+        return IDKM_ERR_CUDA;
+      }
+    ctx->host_streams_ok = true;
+  }
   char* base = static_cast<char*>(ctx->hbuf);
   float* dW_ = reinterpret_cast<float*>(base);
   float* dG = reinterpret_cast<float*>(base + wbytes);
   float* dWq = reinterpret_cast<float*>(base + 2 * wbytes);
   float* ddW = reinterpret_cast<float*>(base + 3 * wbytes);
-  float* dC0 = reinterpret_cast<float*>(base + 4 * wbytes);
-  float* dC = reinterpret_cast<float*>(base + 4 * wbytes + cbytes);
-  float* ddC = reinterpret_cast<float*>(base + 4 * wbytes + 2 * cbytes);
-  void* ws = base + 4 * wbytes + 3 * cbytes;
-  cudaStream_t s = 0;
+  float* ddWj = reinterpret_cast<float*>(base + 4 * wbytes);
+  float* dC0 = reinterpret_cast<float*>(base + 5 * wbytes);
+  float* dC = reinterpret_cast<float*>(base + 5 * wbytes + cbytes);
+  float* ddC = reinterpret_cast<float*>(base + 5 * wbytes + 2 * cbytes);
+  float* ddCj = reinterpret_cast<float*>(base + 5 * wbytes + 3 * cbytes);
+  void* ws = base + 5 * wbytes + 4 * cbytes;
+  cudaStream_t s = ctx->hs_compute, sc = ctx->hs_copy;
   const size_t wn = sizeof(float) * (size_t)m * d, cn = sizeof(float) * (size_t)n_layers * k * d;
-  if (cudaMemcpyAsync(dW_, W_host, wn, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(dC0, C0_host, cn, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-      cudaMemcpyAsync(dG, dWq_host, wn, cudaMemcpyHostToDevice, s) != cudaSuccess)
-    return IDKM_ERR_CUDA;
+#define IDKM_TRY(call) do { if ((call) != cudaSuccess) { (void)cudaGetLastError(); cudaStreamSynchronize(s); cudaStreamSynchronize(sc); return IDKM_ERR_CUDA; } } while (0)
+  // W and C0 go first on the compute stream; the upstream gradient is uploaded on the copy stream while the forward
+  // loop runs (it is first read by the backward)
+  IDKM_TRY(cudaMemcpyAsync(dW_, W_host, wn, cudaMemcpyHostToDevice, s));
+  IDKM_TRY(cudaMemcpyAsync(dC0, C0_host, cn, cudaMemcpyHostToDevice, s));
+  IDKM_TRY(cudaMemcpyAsync(dG, dWq_host, wn, cudaMemcpyHostToDevice, sc));
+  IDKM_TRY(cudaEventRecord(ctx->hev[0], sc));
   int rc = idkm_forward_batched(ctx, dW_, layer_offsets, n_layers, d, dC0, k, tau, tol, max_iter, dC, nullptr,
                                 Wq_out_host ? dWq : nullptr, ws, ws_bytes, s);
-  if (rc != IDKM_OK) return rc;
+  if (rc != IDKM_OK) { cudaStreamSynchronize(s); cudaStreamSynchronize(sc); return rc; }
+  // C and Wq go back on the copy stream while the backward runs
+  IDKM_TRY(cudaEventRecord(ctx->hev[1], s));
+  IDKM_TRY(cudaStreamWaitEvent(sc, ctx->hev[1], 0));
+  IDKM_TRY(cudaMemcpyAsync(C_out_host, dC, cn, cudaMemcpyDeviceToHost, sc));
+  if (Wq_out_host) IDKM_TRY(cudaMemcpyAsync(Wq_out_host, dWq, wn, cudaMemcpyDeviceToHost, sc));
+  IDKM_TRY(cudaStreamWaitEvent(s, ctx->hev[0], 0));
+  if (also_jfb) {
+    rc = idkm_backward(ctx, dG, IDKM_JFB, 0.f, 0, 1.f, dW_jfb_out_host ? ddWj : nullptr, dC_jfb_out_host ? ddCj : nullptr,
+                       ws, ws_bytes, s);
+    if (rc != IDKM_OK) { cudaStreamSynchronize(s); cudaStreamSynchronize(sc); return rc; }
+    IDKM_TRY(cudaEventRecord(ctx->hev[2], s));
+    IDKM_TRY(cudaStreamWaitEvent(sc, ctx->hev[2], 0));
+    if (dW_jfb_out_host) IDKM_TRY(cudaMemcpyAsync(dW_jfb_out_host, ddWj, wn, cudaMemcpyDeviceToHost, sc));
+    if (dC_jfb_out_host) IDKM_TRY(cudaMemcpyAsync(dC_jfb_out_host, ddCj, cn, cudaMemcpyDeviceToHost, sc));
+  }
   rc = idkm_backward(ctx, dG, mode, adj_tol, adj_max_iter, alpha, dW_out_host ? ddW : nullptr,
                      dC_out_host ? ddC : nullptr, ws, ws_bytes, s);
-  if (rc != IDKM_OK) return rc;
-  if (cudaMemcpyAsync(C_out_host, dC, cn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
-  if (Wq_out_host && cudaMemcpyAsync(Wq_out_host, dWq, wn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
-  if (dW_out_host && cudaMemcpyAsync(dW_out_host, ddW, wn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
-  if (dC_out_host && cudaMemcpyAsync(dC_out_host, ddC, cn, cudaMemcpyDeviceToHost, s) != cudaSuccess) return IDKM_ERR_CUDA;
-  if (cudaStreamSynchronize(s) != cudaSuccess) return IDKM_ERR_CUDA;
+  if (rc != IDKM_OK) { cudaStreamSynchronize(s); cudaStreamSynchronize(sc); return rc; }
+  if (dW_out_host) IDKM_TRY(cudaMemcpyAsync(dW_out_host, ddW, wn, cudaMemcpyDeviceToHost, s));
+  if (dC_out_host) IDKM_TRY(cudaMemcpyAsync(dC_out_host, ddC, cn, cudaMemcpyDeviceToHost, s));
+#undef IDKM_TRY
+  if (cudaStreamSynchronize(sc) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) return IDKM_ERR_CUDA;
   if (info_out) return idkm_get_info(ctx, info_out);
   return IDKM_OK;
+}
+
+int idkm_quantize_host(idkm_ctx* ctx, const float* W_host, const int64_t* layer_offsets, int n_layers, int d,
+                       const float* C0_host, int k, float tau, float tol, int max_iter, const float* dWq_host,
+                       idkm_mode mode, float adj_tol, int adj_max_iter, float alpha, float* C_out_host,
+                       float* Wq_out_host, float* dW_out_host, float* dC_out_host, idkm_info* info_out) {
+  return idkm_quantize_host_ex(ctx, W_host, layer_offsets, n_layers, d, C0_host, k, tau, tol, max_iter, dWq_host, mode,
+                               adj_tol, adj_max_iter, alpha, C_out_host, Wq_out_host, dW_out_host, dC_out_host, nullptr,
+                               nullptr, info_out);
 }
 
 int idkm_set_timing(idkm_ctx* ctx, int enable) {
@@ -853,6 +910,21 @@ int idkm_count_busy_tickets(idkm_ctx* ctx, int* count_out) {
 }
 
 int64_t idkm_launch_count(const idkm_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int idkm_describe_path(int d, int k, int adj_max_iter, int adjoint_method, int* out) {
+  if (!out) return IDKM_ERR_NULL;
+  if (d_index(d) < 0 || k < 1 || k > IDKM_MAX_K) return IDKM_ERR_UNSUPPORTED;
+  const int fs = pick_family(STEP, d, k), fa = pick_family(ADJ, d, k), fj = pick_family(JACOBIAN, d, k);
+  if (fs < 0 || fa < 0) return IDKM_ERR_UNSUPPORTED;
+  out[0] = kernel_entry(STEP, d, fs)->kpl;
+  out[1] = kernel_entry(STEP, d, fs)->lpw;
+  out[2] = kernel_entry(ADJ, d, fa)->kpl;
+  out[3] = kernel_entry(ADJ, d, fa)->lpw;
+  const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, d, fj)->plen > JAC_SMALL_PLEN_MAX;
+  const bool explicit_jac = adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS);
+  out[4] = (adj_max_iter <= 0) ? 0 : (explicit_jac ? (jac_tile ? 2 : 1) : 0);
+  return IDKM_OK;
+}
 
 const char* idkm_status_string(int status) {
   switch (status) {

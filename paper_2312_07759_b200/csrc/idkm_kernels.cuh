@@ -552,9 +552,10 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   // the FMA pipe, and the step came out slower, so the arithmetic below is scalar.)
   float2 c2[KH][D];                // owned centroids
   // u_j / S_j (0 for a dead cluster) and kap_j = (u_j / S_j) . F(C_T, W)_j, so that p_ij = (u_j / S_j) . w_i - kap_j.
-  // The full-warp layouts keep them in shared memory ([t][lane] order: conflict-free), the others in registers:
-  // with 8 centroids per lane at two blocks per SM the registers do not hold them without spilling.
-  constexpr bool US_SMEM = NEED_U && (LPW == 32);
+  // The full-warp layouts and the 16-centroids-per-lane layout keep them in shared memory ([t][lane] order:
+  // conflict-free), the others in registers: with 8 centroids per lane at two blocks per SM, or with 16 per lane, the
+  // registers do not hold them without spilling.
+  constexpr bool US_SMEM = NEED_U && (LPW == 32 || KPL == 16);
   float us[(NEED_U && !US_SMEM) ? KPL : 1][D];
   float kap[(NEED_U && !US_SMEM) ? KPL : 1];
   __shared__ __align__(16) float us_sm[US_SMEM ? KPL * LPW * D : 4];
@@ -1000,13 +1001,13 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
     } else {
       // group-per-weight: the group reads one staged row at a time (a shared-memory broadcast)
       const long long gbase = tbase + (long long)grp * WPG;
-#pragma unroll WUNROLL
-      for (int t = 0; t < WPG; ++t) {
-        const long long loc = gbase + t;
-        const bool ok = (loc < rows);
-        const long long grow = row0 + (ok ? loc : 0);
+      // rows of this group's share of the tile that exist (the last tile of a layer may be ragged): one 32-bit
+      // count per tile, so that the row loop carries no 64-bit arithmetic (the backward kernels sit at their
+      // register limit and would otherwise recompute row indices and staging addresses for every row)
+      const long long left = rows - gbase;
+      const int nvalid = left >= WPG ? WPG : (left > 0 ? (int)left : 0);
+      auto one_row = [&](int t, bool ok, const float* ws, const float* gs, const float2* ls) {
         float w[D], gi[D], outv[D];
-        const float* ws = wstage + (grp * WPG + t) * D;
         if constexpr (D == 4) {
           const float4 x = *reinterpret_cast<const float4*>(ws);
           w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
@@ -1019,7 +1020,6 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
 #pragma unroll
         for (int a = 0; a < D; ++a) gi[a] = 0.f;
         if constexpr (NEED_G) {
-          const float* gs = gstage + (grp * WPG + t) * D;
           if constexpr (D == 4) {
             const float4 y = *reinterpret_cast<const float4*>(gs);
             gi[0] = y.x; gi[1] = y.y; gi[2] = y.z; gi[3] = y.w;
@@ -1032,9 +1032,12 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         }
         float2 rstat = make_float2(0.f, 0.f);
         if constexpr (ROWSTAT_R) {
-          if (ok) rstat = lstage[grp * WPG + t];
+          rstat = *ls;
+          if (!ok) rstat.y = 0.f;      // a zero normaliser switches the row off
         }
         if constexpr (ROWSTAT_W) stage_slot = grp * WPG + t;
+        long long grow = 0;
+        if constexpr (MODE == FINAL || MODE == SCATTER) grow = row0 + gbase + (ok ? t : 0);
         process(w, gi, ok, grow, outv, rstat);
         if constexpr (MODE == FINAL || MODE == SCATTER) {
           float* dst = (MODE == FINAL) ? p.Wq : p.dW;
@@ -1043,6 +1046,24 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
             else if constexpr (D == 2) *reinterpret_cast<float2*>(dst + grow * 2) = make_float2(outv[0], outv[1]);
             else dst[grow] = outv[0];
           }
+        }
+      };
+      if constexpr (MODE == STEP) {
+        // the forward step measured 10 % slower with the loop below (two rows in flight interleave less well)
+#pragma unroll WUNROLL
+        for (int t = 0; t < WPG; ++t)
+          one_row(t, gbase + t < rows, wstage + (grp * WPG + t) * D, gstage + (NEED_G ? (grp * WPG + t) * D : 0), lstage + (ROWSTAT_R ? grp * WPG + t : 0));
+      } else {
+        // running pointers: one add per staged array and row
+        const float* ws = wstage + grp * (WPG * D);
+        const float* gs = gstage + (NEED_G ? grp * (WPG * D) : 0);
+        const float2* ls = lstage + (ROWSTAT_R ? grp * WPG : 0);
+#pragma unroll WUNROLL
+        for (int t = 0; t < WPG; ++t) {
+          one_row(t, t < nvalid, ws, gs, ls);
+          ws += D;
+          if constexpr (NEED_G) gs += D;
+          if constexpr (ROWSTAT_R) ls += 1;
         }
       }
       if constexpr (ROWSTAT_W) {

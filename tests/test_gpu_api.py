@@ -72,6 +72,34 @@ def test_quantize_host_matches_oracle():
     assert ctx.launches == 2 * (1 + 1 + 1 + 1 + 6 + 1)   # init, the single-launch forward loop, final, g, adjoint, dW
 
 
+def test_quantize_host_with_both_gradients_from_one_forward():
+    """idkm_quantize_host_ex: the implicit and the Jacobian-free gradients of one forward, copies overlapped with the
+    kernels on the ctx's own two streams (pinned and pageable host buffers both work)."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(120000, 4, 64, 0.012, std=0.03, seed=9, max_iter=8, adj_max_iter=5, init="rows")
+    ref_i, ref_j = oracle_run(wl, mode="implicit"), oracle_run(wl, mode="jfb")
+    ctx = B.Context()
+    for pinned in (False, True):
+        W, C0, G = wl.W, wl.C0, wl.G
+        if pinned:
+            W, C0, G = (torch.from_numpy(x).pin_memory().numpy() for x in (wl.W, wl.C0, wl.G))
+        C, Wq, dW, dC, infos, dWj, dCj = ctx.quantize_host(W, C0, G, wl.tau, 0.0, wl.max_iter, B.IMPLICIT, 0.0,
+                                                           wl.adj_max_iter, 1.0, also_jfb=True)
+        assert infos[0].status == 0 and infos[0].fwd_iters == 8 and infos[0].adj_iters == 5
+        assert_close(C, ref_i["C"], TOL_C, "C")
+        assert_close(Wq, ref_i["Wq"], TOL_C, "Wq")
+        assert_close(dW, ref_i["dW"], TOL_GRAD, "dW implicit")
+        assert_close(dC, ref_i["dC"], TOL_GRAD, "dC implicit")
+        assert_close(dWj, ref_j["dW"], TOL_GRAD, "dW jfb")
+        assert_close(dCj, ref_j["dC"], TOL_GRAD, "dC jfb")
+    out = B.describe_path(4, 64, 5)
+    assert out["adjoint_route"] == "fused passes" and out["adjoint_layout"][0] * out["adjoint_layout"][1] >= 64
+    assert B.describe_path(1, 4, 30)["adjoint_route"] == "explicit Jacobian in registers"
+    assert B.describe_path(1, 16, 30)["adjoint_route"] == "explicit Jacobian in tiles"
+    assert B.describe_path(1, 16, 4)["adjoint_route"] == "fused passes"
+
+
 def test_non_default_stream():
     import torch
     from paper_2312_07759_b200 import binding as B
