@@ -241,6 +241,23 @@ int idkm_step_noalloc_status(int* status_host_out, void* cuda_stream);
 int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
 
 /*
+ * Which distance the softmax of the E-step takes.  0 (default): the Euclidean norm, D_ij = ||w_i - c_j||_2, as
+ * Algorithm 1 (step 3) and the equation for a_j(w_i, C) state it.  1: its square, D_ij = ||w_i - c_j||_2^2, the
+ * distance in which the clustering objectives are written (the k-means objective of Section 3.1 and the soft
+ * objective of Section 3.2); A_ij is then the posterior of an equal-weight mixture of isotropic Gaussians of variance
+ * tau / 2, the gradient dD_ij/dw_i = 2 (w_i - c_j) has no kink at w_i = c_j, and a pair costs one special-function
+ * operation (the exponential) instead of two.  Everything else -- F, Wq, the implicit and Jacobian-free gradients,
+ * statuses -- is defined as above with that D.  Applies to the following idkm_forward* / idkm_backward /
+ * idkm_quantize_host* calls of the ctx; a backward must follow a forward made with the same setting (else
+ * IDKM_ERR_ORDER).  In this setting every forward iteration is one launch per iteration of the fused fp32 step
+ * (no one-launch loop, no fp64 step for collapsing layers) and the implicit backward always iterates fused passes.
+ * A temperature schedule (start warm, end cold, as the paper's closing section suggests) is a sequence of forward
+ * calls in which each call's C0 is the previous call's C_out.
+ * Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_PARAM.
+ */
+int idkm_set_distance(idkm_ctx* ctx, int squared);
+
+/*
  * Hard assignment, q(w) = argmin_c ||w - c|| (Section 3.1: the map the soft quantiser r_tau of the forward tends
  * to as tau -> 0) -- the codes and dequantised weights of the trained layer.  For every row i of W [m][d] (DEVICE,
  * fp32) the index of the nearest row of C [k][d] (DEVICE, fp32; squared distances in fp32, ties to the lowest index)

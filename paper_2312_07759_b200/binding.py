@@ -71,6 +71,8 @@ lib.idkm_set_test_hooks.argtypes = [_vp, C.c_int, C.c_int64]
 lib.idkm_set_test_hooks.restype = C.c_int
 lib.idkm_count_busy_tickets.argtypes = [_vp, C.POINTER(C.c_int)]
 lib.idkm_count_busy_tickets.restype = C.c_int
+lib.idkm_set_distance.argtypes = [_vp, C.c_int]
+lib.idkm_set_distance.restype = C.c_int
 lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
 lib.idkm_set_adjoint_method.restype = C.c_int
 lib.idkm_get_history.argtypes = [_vp, C.c_int, C.c_int, C.POINTER(C.c_float), C.c_int, C.POINTER(C.c_int)]
@@ -295,6 +297,12 @@ class Context:
         _check(rc)
         self.n_layers = L
         return Cout, Wq, dW, dC, list(infos)
+
+    def set_distance(self, squared: bool) -> None:
+        """``idkm_set_distance``: False = Euclidean distance in the softmax (Algorithm 1), True = its square."""
+        _check(lib.idkm_set_distance(self._h, 1 if squared else 0))
+        self._keep = None if squared != getattr(self, "_squared", False) else self._keep
+        self._squared = bool(squared)
 
     def set_adjoint_method(self, method: int) -> None:
         """0: explicit Jacobian for k*d <= 8 (default); 1: always one fused pass per adjoint step."""

@@ -20,6 +20,11 @@ extern const KernelEntry k_table_final[3][N_FAMILY];
 extern const KernelEntry k_table_grad[3][N_FAMILY];
 extern const KernelEntry k_table_adj[3][N_FAMILY];
 extern const KernelEntry k_table_scatter[3][N_FAMILY];
+extern const KernelEntry k_table_step_sq[3][N_FAMILY];
+extern const KernelEntry k_table_final_sq[3][N_FAMILY];
+extern const KernelEntry k_table_grad_sq[3][N_FAMILY];
+extern const KernelEntry k_table_adj_sq[3][N_FAMILY];
+extern const KernelEntry k_table_scatter_sq[3][N_FAMILY];
 extern const KernelEntry k_table_step_precise[3][N_FAMILY];
 extern const KernelEntry k_table_jacobian[3][N_FAMILY];
 extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY];
@@ -28,7 +33,7 @@ extern const DualEntry k_table_dual[3][2];
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
                                   double inv_tau, unsigned int* gtickets, int n_groups, unsigned int* sync,
-                                  unsigned int* gtickets64, int n_groups64) {
+                                  unsigned int* gtickets64, int n_groups64, int squared) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   for (int o = i; o < n_groups; o += gridDim.x * blockDim.x) gtickets[o] = 0u;
   for (int o = i; o < n_groups64; o += gridDim.x * blockDim.x) gtickets64[o] = 0u;
@@ -38,7 +43,8 @@ __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0,
     s.fwd_done = 0; s.fwd_iters = 0; s.fwd_res = 0.f; s.dead = 0;
     s.adj_done = 0; s.adj_iters = 0; s.adj_res = 0.f; s.status = ST_OK;
     s.ticket = 0u; s.adj_up = 0; s.adj_prev = 3.0e38f;
-    for (int q = 0; q < 3; ++q) s.pad[q] = 0;
+    s.g_norm = 0.f;
+    for (int q = 0; q < 2; ++q) s.pad[q] = 0;
     // bounding box of the starting centroids decides which step kernel takes the layer first
     double box2 = 0.0;
     for (int a = 0; a < d; ++a) {
@@ -50,7 +56,7 @@ __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0,
       }
       box2 += (hi - lo) * (hi - lo);
     }
-    s.precise[0] = s.precise[1] = (sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
+    s.precise[0] = s.precise[1] = (!squared && sqrt(box2) * inv_tau <= PRECISE_SPAN) ? 1 : 0;
     st[i] = s;
   }
   if (C0 != C)
@@ -58,6 +64,20 @@ __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0,
 }
 
 static int d_index(int d) { return d == 1 ? 0 : (d == 2 ? 1 : (d == 4 ? 2 : -1)); }
+
+// The squared-distance variant of a fused pass (same layouts, same tile and partial sizes as kernel_entry's).
+static const KernelEntry* kernel_entry_sq(int mode, int d, int family) {
+  const int di = d_index(d);
+  if (di < 0 || family < 0 || family >= N_FAMILY) return nullptr;
+  switch (mode) {
+    case STEP: return &k_table_step_sq[di][family];
+    case FINAL: return &k_table_final_sq[di][family];
+    case GRAD: return &k_table_grad_sq[di][family];
+    case ADJ: return &k_table_adj_sq[di][family];
+    case SCATTER: return &k_table_scatter_sq[di][family];
+  }
+  return nullptr;
+}
 
 const KernelEntry* kernel_entry(int mode, int d, int family) {
   const int di = d_index(d);
@@ -227,7 +247,7 @@ struct idkm_ctx {
   float tau;
   long long row_off[MAX_LAYERS + 1];
   cudaStream_t stream;
-  int occupancy[N_MODES][3][N_FAMILY];   // cached blocks/SM per kernel, 0 = not queried
+  int occupancy[2][N_MODES][3][N_FAMILY];   // cached blocks/SM per kernel ([1]: squared-distance variants), 0 = not queried
   // device buffers, streams and events of the host-pointer entry point
   void* hbuf;
   size_t hbuf_bytes;
@@ -238,6 +258,7 @@ struct idkm_ctx {
   bool timing;
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
+  int squared;          // 1: squared-distance variant (idkm_set_distance)
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
   int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never;
                         // 2: never, and the fp32 and fp64 steps of an iteration are always two launches
@@ -259,11 +280,18 @@ static void mark(idkm_ctx* ctx, int i) {
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The kernel that runs a pass for this ctx: the squared-distance variant of the fused passes when the ctx asks for it.
+static const KernelEntry* ctx_entry(const idkm_ctx* ctx, int mode, int family) {
+  if (ctx->squared && mode <= SCATTER) return kernel_entry_sq(mode, ctx->d, family);
+  return kernel_entry(mode, ctx->d, family);
+}
+
 static int blocks_per_sm(idkm_ctx* ctx, int mode, int d, int family) {
-  int& slot = ctx->occupancy[mode][d_index(d)][family];
+  const bool sq = ctx->squared && mode <= SCATTER;
+  int& slot = ctx->occupancy[sq ? 1 : 0][mode][d_index(d)][family];
   if (slot == 0) {
     int n = 0;
-    const KernelEntry* e = kernel_entry(mode, d, family);
+    const KernelEntry* e = sq ? kernel_entry_sq(mode, d, family) : kernel_entry(mode, d, family);
     // static + dynamic shared memory can exceed the 48 KB default: raise the limit before asking for the occupancy
     if (e->dyn_smem > 0) (void)cudaFuncSetAttribute(e->func, cudaFuncAttributeMaxDynamicSharedMemorySize, e->dyn_smem);
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, e->func, BLOCK, e->dyn_smem) != cudaSuccess || n < 1) {
@@ -329,6 +357,7 @@ static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p)
   p->scale = (float)(1.4426950408889634 / (double)ctx->tau);
   p->alpha = 1.f;
   p->k = ctx->k;
+  p->squared = ctx->squared;
 }
 
 // Loops with a tolerance are queued in chunks of RUN_CHUNK iterations.  After each chunk the host peeks at the pinned
@@ -368,10 +397,10 @@ struct RunAhead {
 // of them (LayerState::precise), the other returns at once for it.
 static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p, int repeat) {
   const int f32 = pick_family(STEP, ctx->d, ctx->k), f64 = pick_family(STEP_PRECISE, ctx->d, ctx->k);
-  const KernelEntry* e32 = kernel_entry(STEP, ctx->d, f32);
+  const KernelEntry* e32 = ctx_entry(ctx, STEP, f32);
   const KernelEntry* e64 = kernel_entry(STEP_PRECISE, ctx->d, f64);
   static const bool dual_off = (getenv("IDKM_NO_DUAL") != nullptr);   // tuning knob: always two launches per iteration
-  const DualEntry* de = (dual_off || ctx->forward_loop == 2) ? nullptr : dual_entry(ctx->d, ctx->k);
+  const DualEntry* de = (dual_off || ctx->forward_loop == 2 || ctx->squared) ? nullptr : dual_entry(ctx->d, ctx->k);
   PassParams q = *p;
   int rc = build_table(ctx, STEP, f32, &p->lt);
   if (rc != IDKM_OK) return rc;
@@ -400,8 +429,11 @@ static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams
       ctx->launches += 1;
     } else {
       if (e32->launch(*p, p->lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
-      if (e64->launch(q, q.lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
-      ctx->launches += 2;
+      ctx->launches += 1;
+      if (!ctx->squared) {   // (the squared-distance variant never hands a layer to the fp64 step)
+        if (e64->launch(q, q.lt.n_blocks, ctx->stream) != cudaSuccess) return IDKM_ERR_CUDA;
+        ctx->launches += 1;
+      }
     }
     if (ra.after(it)) break;
   }
@@ -421,7 +453,7 @@ constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM c
 // Returns IDKM_OK after queueing the loop, 1 if this problem should take the launch-per-iteration path.
 static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p, int max_iter) {
   static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
-  if (env_off || ctx->forward_loop != 0 || ctx->n_layers != 1 || max_iter < 2) return 1;
+  if (env_off || ctx->forward_loop != 0 || ctx->n_layers != 1 || max_iter < 2 || ctx->squared) return 1;
   const int di = d_index(ctx->d);
   int f = -1;
   for (int q = 0; q < N_SMALL_FAMILY; ++q)
@@ -475,7 +507,7 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
 
 static int launch_pass(idkm_ctx* ctx, int mode, PassParams* p, int repeat) {
   const int f = pick_family(mode, ctx->d, ctx->k);
-  const KernelEntry* e = kernel_entry(mode, ctx->d, f);
+  const KernelEntry* e = ctx_entry(ctx, mode, f);
   const int rc = build_table(ctx, mode, f, &p->lt);
   if (rc != IDKM_OK) return rc;
   RunAhead ra;
@@ -590,7 +622,7 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
                                                                                      p.inv_tau_d, p.gtickets, wl.max_groups,
                                                                                      reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + wl.off_sync),
                                                                                      reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + wl.off_gtickets64),
-                                                                                     wl.max_groups64);
+                                                                                     wl.max_groups64, ctx->squared);
   if (cudaGetLastError() != cudaSuccess) return IDKM_ERR_CUDA;
   ++ctx->launches;
   mark(ctx, 1);
@@ -647,7 +679,8 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   const bool solve = (mode == IDKM_IMPLICIT && adj_max_iter > 0);
   const int fj = pick_family(JACOBIAN, ctx->d, ctx->k);
   const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, ctx->d, fj)->plen > JAC_SMALL_PLEN_MAX;
-  const bool explicit_jac = ctx->adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS);
+  // (the explicit-Jacobian kernels are written for the Euclidean distance: the squared variant takes the fused passes)
+  const bool explicit_jac = ctx->adjoint_method == 0 && !ctx->squared && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS);
   // the per-row softmax reference and normaliser are kept only if fused adjoint passes follow
   if (!solve || explicit_jac) p.rowstat = nullptr;
   mark(ctx, 4);
@@ -863,6 +896,14 @@ int idkm_get_history(idkm_ctx* ctx, int which, int layer, float* host_out, int c
   if (n > 0 && cudaMemcpy(host_out, ws + off, sizeof(float) * (size_t)n, cudaMemcpyDeviceToHost) != cudaSuccess)
     return IDKM_ERR_CUDA;
   *n_out = n;
+  return IDKM_OK;
+}
+
+int idkm_set_distance(idkm_ctx* ctx, int squared) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (squared != 0 && squared != 1) return IDKM_ERR_PARAM;
+  if (ctx->squared != squared) ctx->have_forward = false;   // a backward must follow a forward of the same variant
+  ctx->squared = squared;
   return IDKM_OK;
 }
 

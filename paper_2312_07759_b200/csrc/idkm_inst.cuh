@@ -28,24 +28,29 @@ static cudaError_t launch_pdl(Kernel kernel, const PassParams& p, int grid, int 
   return cudaLaunchKernelEx(&cfg, kernel, p);
 }
 
-template <int MODE, int D, int KPL, int LPW>
+template <int MODE, int D, int KPL, int LPW, bool SQ>
 static cudaError_t launch_one(const PassParams& p, int grid, cudaStream_t stream) {
   constexpr int DYN = PassCfg<MODE, D, KPL, LPW>::DYN_SMEM;
   static bool configured = false;   // static + dynamic shared memory may exceed the 48 KB default
   if (!configured) {
-    const cudaError_t rc = cudaFuncSetAttribute(idkm_pass<MODE, D, KPL, LPW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                DYN > 0 ? DYN : 1);
+    const cudaError_t rc = cudaFuncSetAttribute(idkm_pass<MODE, D, KPL, LPW, SQ>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, DYN > 0 ? DYN : 1);
     if (rc != cudaSuccess) return rc;
     configured = true;
   }
-  return launch_pdl(idkm_pass<MODE, D, KPL, LPW>, p, grid, DYN, stream);
+  return launch_pdl(idkm_pass<MODE, D, KPL, LPW, SQ>, p, grid, DYN, stream);
 }
 
-#define IDKM_ENTRY(MODE, D, KPL, LPW)                                                             \
-  {                                                                                               \
-    &launch_one<MODE, D, KPL, LPW>, (const void*)&idkm_pass<MODE, D, KPL, LPW>, KPL, LPW,         \
-        PassCfg<MODE, D, KPL, LPW>::TILE, PassCfg<MODE, D, KPL, LPW>::PLEN,                       \
-        PassCfg<MODE, D, KPL, LPW>::DYN_SMEM                                                      \
+// IDKM_SQ selects which variant a translation unit instantiates: the Euclidean distance of Algorithm 1 (default) or
+// the squared distance (the *_sq.cu units define it as true before including this header).
+#ifndef IDKM_SQ
+#define IDKM_SQ false
+#endif
+#define IDKM_ENTRY(MODE, D, KPL, LPW)                                                                       \
+  {                                                                                                         \
+    &launch_one<MODE, D, KPL, LPW, IDKM_SQ>, (const void*)&idkm_pass<MODE, D, KPL, LPW, IDKM_SQ>, KPL, LPW, \
+        PassCfg<MODE, D, KPL, LPW>::TILE, PassCfg<MODE, D, KPL, LPW>::PLEN,                                 \
+        PassCfg<MODE, D, KPL, LPW>::DYN_SMEM                                                                \
   }
 
 template <int D, int KPL, int LPW>
@@ -87,6 +92,15 @@ static cudaError_t launch_jacobian(const PassParams& p, int grid, cudaStream_t s
     IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
         IDKM_ENTRY(MODE, D, 8, 2), IDKM_ENTRY(MODE, D, 8, 4), IDKM_ENTRY(MODE, D, 8, 8),          \
         IDKM_ENTRY(MODE, D, 8, 16), IDKM_ENTRY(MODE, D, 8, 32), IDKM_ENTRY(MODE, D, 8, 32)        \
+  }
+// The adjoint step's last entry is the half-warp layout with 16 centroids per lane (one block of 8 warps per SM,
+// 254 registers): half the per-row overhead and one shuffle stage fewer per pair than 8 centroids on a full warp, and
+// the registers keep w - c_j from the distance to the accumulation.
+#define IDKM_ADJ_ROW(D)                                                                           \
+  {                                                                                               \
+    IDKM_ENTRY(ADJ, D, 2, 1), IDKM_ENTRY(ADJ, D, 4, 1), IDKM_ENTRY(ADJ, D, 8, 1),                 \
+        IDKM_ENTRY(ADJ, D, 8, 2), IDKM_ENTRY(ADJ, D, 8, 4), IDKM_ENTRY(ADJ, D, 8, 8),             \
+        IDKM_ENTRY(ADJ, D, 8, 16), IDKM_ENTRY(ADJ, D, 8, 32), IDKM_ENTRY(ADJ, D, 16, 16)          \
   }
 
 }  // namespace idkm

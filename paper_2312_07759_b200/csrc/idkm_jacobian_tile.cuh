@@ -132,6 +132,15 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
       const double al = (double)p.alpha;
       int it = 0, up = 0, status = st->status, done = 0;
       float res = 0.f, prev = 3.0e38f;
+      double g2 = 0.0;
+#pragma unroll
+      for (int h = 0; h < QPL; ++h) {
+        const int q = lane + 32 * h;
+        if (q < n) g2 += gs[q] * gs[q];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) g2 += __shfl_xor_sync(0xffffffffu, g2, o);
+      const double u2_limit = ADJ_GROWTH_LIMIT * ADJ_GROWTH_LIMIT * g2;
       while (it < p.max_iter && !done) {
         double un[QPL];
         double num = 0.0, den = 0.0, badv = 0.0;
@@ -167,7 +176,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
         if (lane == 0 && it <= HIST_CAP) p.hist_adj[(size_t)l * HIST_CAP + it - 1] = res;
         up = (res > prev) ? up + 1 : 0;
         prev = res;
-        if (badv > 0.0 || up >= 10) {
+        if (badv > 0.0 || up >= 10 || den > u2_limit) {
           status = ST_DIVERGED;
           done = 1;
         } else if (p.tol > 0.f && res < p.tol) {

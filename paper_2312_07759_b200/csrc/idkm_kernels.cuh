@@ -35,6 +35,11 @@ constexpr int RED_SINGLE_MAX = 64;
 // weight differ by less than PRECISE_SPAN and the centroid update is decided by attention differences far below
 // fp32 resolution (w - c_j rounds away the differences between the c_j).  Such layers step in fp64.
 constexpr double PRECISE_SPAN = 0.0625;
+// A converging adjoint iteration u <- alpha (J^T u + g) + (1 - alpha) u stays below ||g|| / (1 - rho); once ||u|| has
+// grown past this multiple of ||g|| the iteration is reported as diverged (Section 4.2: "if we see the iteration
+// diverge, we start over and divide alpha by 2").  A residual that grows 10 steps running, or a non-finite u, counts
+// as well; a spiralling (complex-eigenvalue) divergence shows only in the norm.
+constexpr double ADJ_GROWTH_LIMIT = 1e6;
 
 enum Mode { STEP = 0, FINAL = 1, GRAD = 2, ADJ = 3, SCATTER = 4, STEP_PRECISE = 5, JACOBIAN = 6 };
 constexpr int N_MODES = 7;
@@ -57,7 +62,9 @@ struct LayerState {   // 64 bytes, one per layer, in the workspace
                      // writes entry (t + 1) & 1 only, so nothing a launch routes by changes while it runs: the fp32
                      // and the fp64 half of the dual step kernel, whose blocks are not ordered against each other,
                      // can never both take (or both skip) a layer.
-  int pad[3];
+  float g_norm;      // ||g||_2 of the last codebook-gradient pass: the adjoint iteration counts as diverged once
+                     // ||u||_2 exceeds ADJ_GROWTH_LIMIT times it
+  int pad[2];
 };
 static_assert(sizeof(LayerState) == 64, "LayerState layout");
 
@@ -98,6 +105,8 @@ struct PassParams {
   int max_iter;       // iteration cap of the loop (for the advisory status)
   int* host_flag;     // device view of a pinned host word, or null: set to call_id once every layer's loop has ended
   int call_id;
+  int squared;        // 1: squared-distance variant; its layers always step in the fp32 kernel (the fp64 step's
+                      // short exponential series is derived for the Euclidean distance)
   int iter;           // index of this forward iteration: a layer is stepped only while fwd_iters == iter, so that
                       // the fp32 and the fp64 step launched for the same iteration never both take it
   LayerTable lt;
@@ -362,6 +371,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
     for (int o = tid; o < k * D; o += BLOCK) {
       const double gv = tot[o];
       if (!(gv == gv) || fabs(gv) > 1e300) bad += 1.0;
+      den += gv * gv;
       p.gvec[(size_t)l * k * D + o] = (float)gv;
       p.u[(size_t)l * k * D + o] = (float)gv;
     }
@@ -421,7 +431,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   if (tid == 0) {
     st->ticket = 0u;
     if constexpr (MODE == STEP) {
-      st->precise[(p.iter + 1) & 1] = (sqrt(box2) * p.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
+      st->precise[(p.iter + 1) & 1] = (!p.squared && sqrt(box2) * p.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
       double dn = sqrt(den);
       if (dn < 1e-300) dn = 1e-300;
       const float res = (float)(sqrt(num) / dn);
@@ -447,6 +457,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
       st->adj_res = 0.f;
       st->adj_up = 0;
       st->adj_prev = 3.0e38f;
+      st->g_norm = (float)sqrt(den);
       if (bad > 0.0) st->status = ST_NONFINITE;
       else if (st->status == ST_DIVERGED) st->status = ST_OK;
     } else if constexpr (MODE == ADJ) {
@@ -460,7 +471,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
       const int up = (res > st->adj_prev) ? st->adj_up + 1 : 0;
       st->adj_up = up;
       st->adj_prev = res;
-      if (bad > 0.0 || up >= 10) {
+      if (bad > 0.0 || up >= 10 || sqrt(den) > ADJ_GROWTH_LIMIT * (double)st->g_norm) {
         st->status = ST_DIVERGED;
         st->adj_done = 1;
       } else if (p.tol > 0.f && res < p.tol) {
@@ -493,7 +504,10 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
 // RELEASE: let the next kernel of the stream be scheduled once this block's rows are done (the caller has already
 // waited for the previous kernel).  The dual step kernel runs this body with RELEASE = false and releases after its
 // second body.
-template <int MODE, int D, int KPL, int LPW, bool RELEASE>
+// SQ: the squared-distance variant, D_ij = ||w_i - c_j||^2 in the softmax (the distance the clustering objectives of
+// Sections 3.1 / 3.2 are written in) and n_ij = dD_ij/dw_i = 2 (w_i - c_j): no square root, no reciprocal square
+// root, no kink at w_i = c_j.
+template <int MODE, int D, int KPL, int LPW, bool RELEASE, bool SQ = false>
 __device__ __forceinline__ void pass_body(const PassParams& p) {
   using Cfg = PassCfg<MODE, D, KPL, LPW>;
   constexpr int NACC = Cfg::NACC;
@@ -637,7 +651,15 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         // above the first half's arithmetic, which cost more registers than the full-warp layout at d = 4 has
         if (US_SMEM && D == 4 && t == KPL / 2) __syncwarp();
         float dist_t, rs_t = 1.f;
-        if constexpr (D == 1) {
+        if constexpr (SQ) {
+          float sq = 0.f;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const float df = w[a] - c_(t, a);
+            sq = fmaf(df, df, sq);
+          }
+          dist_t = sq;
+        } else if constexpr (D == 1) {
           dist_t = fabsf(w[0] - c_(t, 0));
         } else {
           float sq = 1e-30f;   // rsqrt stays finite when w == c (n_ij = 0 then)
@@ -655,11 +677,11 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         for (int a = 0; a < D; ++a) v = fmaf(us_(t, a), w[a], v);
         z[t] = v;
         lzp[t & 3] = fmaf(et0, v, lzp[t & 3]);
-        ers[t] = (D > 1) ? et0 * rs_t : et0;
+        ers[t] = (D > 1 && !SQ) ? et0 * rs_t : et0;
       }
       const float rr = rstat.y;
       const float zbar = group_sum<LPW>((lzp[0] + lzp[1]) + (lzp[2] + lzp[3])) * rr;
-      const float rt = rr * p.inv_tau;
+      const float rt = rr * (SQ ? 2.f * p.inv_tau : p.inv_tau);   // squared distance: n_ij = 2 (w_i - c_j)
       const float nzr = -zbar * rt;
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
@@ -668,7 +690,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         for (int a = 0; a < D; ++a) {
           const float df = w[a] - c_(t, a);
           float n;
-          if constexpr (D == 1) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
+          if constexpr (D == 1 && !SQ) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
           else n = df;
           acc_(t, a) = fmaf(et, n, acc_(t, a));
         }
@@ -676,7 +698,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
       return;
     }
     float dist[KPL];
-    float rs[(D > 1 && !FWD) ? KPL : 1];
+    float rs[(D > 1 && !FWD && !SQ) ? KPL : 1];
     (void)rs; (void)dist;
     float e[KPL];
     float lmin = 3.0e38f;
@@ -685,7 +707,15 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
     {
 #pragma unroll
       for (int t = 0; t < KPL; ++t) {
-        if constexpr (D == 1) {
+        if constexpr (SQ) {
+          float sq = 0.f;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const float df = w[a] - c_(t, a);
+            sq = fmaf(df, df, sq);
+          }
+          dist[t] = sq;
+        } else if constexpr (D == 1) {
           dist[t] = fabsf(w[0] - c_(t, 0));
         } else {
           // the backward passes start the square at 1e-30 so that rsqrt stays finite when w == c (n_ij = 0 then)
@@ -769,7 +799,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         lzp[t & 3] = fmaf(e[t], v, lzp[t & 3]);
       }
       const float zbar = group_sum<LPW>((lzp[0] + lzp[1]) + (lzp[2] + lzp[3])) * r;
-      const float rt = r * p.inv_tau;
+      const float rt = r * (SQ ? 2.f * p.inv_tau : p.inv_tau);   // squared distance: n_ij = 2 (w_i - c_j)
       const float nzr = -zbar * rt;
       float dwl[D];
 #pragma unroll
@@ -778,12 +808,12 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
       for (int t = 0; t < KPL; ++t) {
         const float at = e[t] * r;                    // A_ij
         float et = e[t] * fmaf(z[t], rt, nzr);        // e_ij(z) / tau = A_ij (z_ij - zbar_i) / tau
-        if constexpr (D > 1) et *= rs[t];             // ... / D_ij, so that et * (w - c) = e_ij(z) n_ij / tau
+        if constexpr (D > 1 && !SQ) et *= rs[t];      // ... / D_ij, so that et * (w - c) = e_ij(z) n_ij / tau
 #pragma unroll
         for (int a = 0; a < D; ++a) {
           const float df = w[a] - c_(t, a);
           float n;
-          if constexpr (D == 1) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
+          if constexpr (D == 1 && !SQ) n = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
           else n = df;
           if constexpr (MODE == GRAD) acc_(t, a) = fmaf(at, gi[a], fmaf(et, n, acc_(t, a)));
           if constexpr (MODE == ADJ) acc_(t, a) = fmaf(et, n, acc_(t, a));
@@ -1091,11 +1121,11 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
 }
 
-template <int MODE, int D, int KPL, int LPW>
+template <int MODE, int D, int KPL, int LPW, bool SQ = false>
 __global__ void __launch_bounds__(BLOCK, PassCfg<MODE, D, KPL, LPW>::MIN_BLOCKS)
 idkm_pass(const __grid_constant__ PassParams p) {
   grid_dependency_sync();
-  pass_body<MODE, D, KPL, LPW, true>(p);
+  pass_body<MODE, D, KPL, LPW, true, SQ>(p);
 }
 
 
@@ -1440,6 +1470,10 @@ __global__ void __launch_bounds__(BLOCK) idkm_jacobian(const __grid_constant__ P
       const double al = (double)p.alpha;
       int it = 0, up = 0, status = st->status, done = 0;
       float res = 0.f, prev = 3.0e38f;
+      double g2 = g * g;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) g2 += __shfl_xor_sync(0xffffffffu, g2, o);
+      const double u2_limit = ADJ_GROWTH_LIMIT * ADJ_GROWTH_LIMIT * g2;
       while (it < p.max_iter && !done) {
         double s = 0.0;
 #pragma unroll
@@ -1461,7 +1495,7 @@ __global__ void __launch_bounds__(BLOCK) idkm_jacobian(const __grid_constant__ P
         if (lane == 0 && it <= HIST_CAP) p.hist_adj[(size_t)l * HIST_CAP + it - 1] = res;
         up = (res > prev) ? up + 1 : 0;
         prev = res;
-        if (badv > 0.0 || up >= 10) {
+        if (badv > 0.0 || up >= 10 || den > u2_limit) {
           status = ST_DIVERGED;
           done = 1;
         } else if (p.tol > 0.f && res < p.tol) {

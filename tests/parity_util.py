@@ -83,26 +83,28 @@ def assert_grad_close(x, ref, what, crossings, tol, tol_kink, record=None):
     return assert_close(x, ref, tol_kink, what + f" ({crossings} kink crossings)", l2_only=True, record=record)
 
 
-def oracle_run(wl, mode="implicit", alpha=1.0, fixed=True, want_A=False, want_dW=True):
+def oracle_run(wl, mode="implicit", alpha=1.0, fixed=True, want_A=False, want_dW=True, squared=False):
     """Oracle forward + final + backward of a single-layer workload (fixed iteration counts when
-    ``fixed``: tolerances disabled)."""
+    ``fixed``: tolerances disabled).  ``squared``: the squared-distance variant."""
     from oracle import idkm_ref as R
     tol = 0.0 if fixed else wl.tol
     adj_tol = 0.0 if fixed else wl.adj_tol
     W, C0, G = wl.W.astype(np.float64), wl.C0.astype(np.float64), wl.G.astype(np.float64)
-    Ct, it, res, dead = R.forward(W, C0, wl.tau, tol, wl.max_iter)
-    Wq, A, S, F = R.final(W, Ct, wl.tau, want_A=want_A)
-    dW, dC, ait, ares = R.backward(W, G, Ct, wl.tau, S, F, mode=mode, alpha=alpha, adj_tol=adj_tol,
-                                   adj_max_iter=wl.adj_max_iter, want_dW=want_dW)
+    with R.squared_distance(squared):
+        Ct, it, res, dead = R.forward(W, C0, wl.tau, tol, wl.max_iter)
+        Wq, A, S, F = R.final(W, Ct, wl.tau, want_A=want_A)
+        dW, dC, ait, ares = R.backward(W, G, Ct, wl.tau, S, F, mode=mode, alpha=alpha, adj_tol=adj_tol,
+                                       adj_max_iter=wl.adj_max_iter, want_dW=want_dW)
     return dict(C=Ct, Wq=Wq, A=A, S=S, F=F, dW=dW, dC=dC, iters=it, res=res, adj_iters=ait, adj_res=ares, dead=dead)
 
 
-def gpu_run(wl, mode="implicit", alpha=1.0, fixed=True, want_A=False, ctx=None, want_dW=True):
+def gpu_run(wl, mode="implicit", alpha=1.0, fixed=True, want_A=False, ctx=None, want_dW=True, squared=False):
     """The same through the C-ABI library on cuda:0."""
     import torch
     from paper_2312_07759_b200 import binding as B
     dev = torch.device("cuda:0")
     ctx = ctx or B.Context()
+    ctx.set_distance(squared)
     W = torch.from_numpy(wl.W).to(dev)
     C0 = torch.from_numpy(wl.C0).to(dev)
     G = torch.from_numpy(wl.G).to(dev)
@@ -118,13 +120,14 @@ def gpu_run(wl, mode="implicit", alpha=1.0, fixed=True, want_A=False, ctx=None, 
                 dW=None if dW is None else dW.cpu().numpy(), dC=dC.cpu().numpy(), info=info, ctx=ctx)
 
 
-def oracle_backward_at(wl, C, mode="implicit", alpha=1.0, want_dW=True):
+def oracle_backward_at(wl, C, mode="implicit", alpha=1.0, want_dW=True, squared=False):
     """Oracle final pass + backward evaluated at the given centroids (fixed adjoint count)."""
     from oracle import idkm_ref as R
     W, G, C = wl.W.astype(np.float64), wl.G.astype(np.float64), np.asarray(C, np.float64)
-    Wq, _, S, F = R.final(W, C, wl.tau)
-    dW, dC, ait, ares = R.backward(W, G, C, wl.tau, S, F, mode=mode, alpha=alpha, adj_tol=0.0,
-                                   adj_max_iter=wl.adj_max_iter, want_dW=want_dW)
+    with R.squared_distance(squared):
+        Wq, _, S, F = R.final(W, C, wl.tau)
+        dW, dC, ait, ares = R.backward(W, G, C, wl.tau, S, F, mode=mode, alpha=alpha, adj_tol=0.0,
+                                       adj_max_iter=wl.adj_max_iter, want_dW=want_dW)
     return dict(C=C, Wq=Wq, dW=dW, dC=dC)
 
 
