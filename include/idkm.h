@@ -55,9 +55,9 @@ extern "C" {
 #define IDKM_ERR_NONFINITE (-9)  /* device: NaN/Inf met in W, C or the sums                     */
 #define IDKM_ERR_NOALLOC_TOO_LARGE (-11) /* idkm_step_noalloc: the problem needs more than the built-in scratch */
 #define IDKM_ERR_TIMEOUT (-12)   /* device: a bounded grid-wide wait of the one-launch forward loop ran out  */
-#define IDKM_ERR_DIVERGED (-10)  /* device: adjoint iteration produced non-finite values or its
-                                    residual grew 10 steps running (Section 4.2: retry with a
-                                    smaller alpha)                                              */
+#define IDKM_ERR_DIVERGED (-10)  /* device: adjoint iteration produced non-finite values, its residual
+                                    grew 10 steps running, or ||u|| passed 1e6 ||g|| (Section 4.2:
+                                    retry with a smaller alpha, see idkm_backward_restart)      */
 
 typedef struct idkm_ctx idkm_ctx; /* opaque; remembers the last forward call for the backward */
 
@@ -237,8 +237,29 @@ int idkm_step_noalloc_status(int* status_host_out, void* cuda_stream);
  * instead of adj_max_iter.  For k d <= 8 always; for 8 < k d <= 64 (the pass costs about ten fused passes) when
  * adj_max_iter >= 16.  Larger codebooks, and shorter iterations, use one fused vector-Jacobian pass per step.
  * 1: always the fused passes.
+ * 2: no iteration where the matrix can be formed (k d <= 64): the same pass forms dF/dC and one warp then solves
+ * (I - (dF/dC)^T) u = g exactly -- the system behind M* = (I - dF/dC)^-1 of Section 4.2 -- by Gaussian elimination
+ * with partial pivoting in fp64; adj_tol, adj_max_iter (> 0) and alpha are ignored, idkm_info reports 0 adjoint
+ * iterations, and a singular system (an eigenvalue 1 of dF/dC) or a non-finite solution reads IDKM_ERR_DIVERGED.
+ * The result is the limit of the iteration where that converges, and is defined (and returned) also where the
+ * iteration would diverge.  Larger codebooks iterate fused passes as with 1.
  */
 int idkm_set_adjoint_method(idkm_ctx* ctx, int method);
+
+/*
+ * Implicit backward with the safeguard of Section 4.2 ("if we see the iteration diverge, we start over and divide
+ * alpha by 2"): runs the codebook gradient and the adjoint iteration of idkm_backward(IDKM_IMPLICIT) with
+ * alpha = alpha0, reads the status (this WAITS for the stream after every attempt), and while any layer reports
+ * IDKM_ERR_DIVERGED starts over from u = g with half the alpha, at most max_halvings times (0 <= max_halvings <= 30).
+ * Then the dL/dW pass and the copy of dC run once, from the last attempt's u.  The alpha of the last attempt and the
+ * number of attempts go to the HOST locations alpha_used_out / attempts_out (may be NULL).  Whether the last attempt
+ * diverged too is in idkm_info.status, as for idkm_backward.  Halving helps where dF/dC has eigenvalues outside the
+ * unit circle whose real part is below 1 (complex pairs occur at centroids that are not yet a fixed point); an
+ * eigenvalue above 1 on the real axis defeats every alpha.  Other arguments and return values as idkm_backward.
+ */
+int idkm_backward_restart(idkm_ctx* ctx, const float* dWq, float adj_tol, int adj_max_iter, float alpha0,
+                          int max_halvings, float* dW_out, float* dC_out, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream, float* alpha_used_out, int* attempts_out);
 
 /*
  * Which distance the softmax of the E-step takes.  0 (default): the Euclidean norm, D_ij = ||w_i - c_j||_2, as
@@ -324,7 +345,8 @@ int idkm_count_busy_tickets(idkm_ctx* ctx, int* count_out);
  * ints to the HOST array out: [0], [1] centroids per lane and lanes per weight-vector of the fused forward step
  * (Algorithm 1, steps 3-5); [2], [3] the same of the fused adjoint step (Section 4.2); [4] how an implicit backward
  * of adj_max_iter steps with idkm_set_adjoint_method = adjoint_method runs the iteration: 0 one fused pass per step,
- * 1 explicit k d x k d matrix held in registers (k d <= 8), 2 explicit matrix in tiles (k d <= 64, from 16 steps).
+ * 1 explicit k d x k d matrix held in registers (k d <= 8), 2 explicit matrix in tiles (k d <= 64, from 16 steps),
+ * 3 exact solve on the explicit matrix (adjoint_method 2, k d <= 64).
  * Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_UNSUPPORTED.  Needs no device.
  */
 int idkm_describe_path(int d, int k, int adj_max_iter, int adjoint_method, int* out);

@@ -315,6 +315,11 @@ void idkm_ref_adjoint_apply(const double *W, int64_t m, int d, const double *C, 
   free(part);
 }
 
+/* One step of the averaged iteration of Section 4.2 on the vector u: un = alpha (J^T u + g) + (1 - alpha) u. */
+static void averaged_step(const double *Ju, const double *g, const double *u, double alpha, int n, double *un) {
+  for (int t = 0; t < n; ++t) un[t] = alpha * (Ju[t] + g[t]) + (1.0 - alpha) * u[t];
+}
+
 /* Adjoint fixed point u = J_C^T u + g, the vector form of M* = (dF/dC) M* + I (Eq. for M*),
  * by the averaged iteration of Section 4.2: u <- alpha (J^T u + g) + (1 - alpha) u, u(0) = g.
  * Stops when the relative change is below adj_tol (adj_tol > 0) or after adj_max_iter steps. */
@@ -329,7 +334,7 @@ void idkm_ref_adjoint_solve(const double *W, int64_t m, int d, const double *C, 
   double res = 0.0;
   while (it < adj_max_iter) {
     idkm_ref_adjoint_apply(W, m, d, C, k, tau, S, F, u, Ju);
-    for (int t = 0; t < n; ++t) un[t] = alpha * (Ju[t] + g[t]) + (1.0 - alpha) * u[t];
+    averaged_step(Ju, g, u, alpha, n, un);
     res = rel_change(un, u, n);
     memcpy(u, un, sizeof(double) * (size_t)n);
     ++it;
@@ -338,6 +343,69 @@ void idkm_ref_adjoint_solve(const double *W, int64_t m, int d, const double *C, 
   if (iters_out) *iters_out = it;
   if (residual_out) *residual_out = res;
   free(Ju);
+}
+
+/* The same iteration under the watch Section 4.2 asks for ("if we see the iteration diverge, we start over and divide
+ * alpha by 2"; the paper gives no criterion, this is the reading taken): the iteration counts as diverged when u is
+ * no longer finite, when the relative change has grown 10 steps running, or when ||u|| has passed 1e6 ||g|| (a
+ * converging iteration stays below ||g|| / (1 - rho)).  Returns 1 if it diverged (u then holds the last iterate),
+ * 0 otherwise. */
+int idkm_ref_adjoint_solve_watched(const double *W, int64_t m, int d, const double *C, int k, double tau,
+                                   const double *S, const double *F, const double *g, double alpha, double adj_tol,
+                                   int adj_max_iter, double *u, int *iters_out, double *residual_out) {
+  const int n = k * d;
+  double *Ju = (double *)malloc(sizeof(double) * (size_t)n * 2);
+  double *un = Ju + n;
+  memcpy(u, g, sizeof(double) * (size_t)n);
+  double g2 = 0.0;
+  for (int t = 0; t < n; ++t) g2 += g[t] * g[t];
+  int it = 0, up = 0, diverged = 0;
+  double res = 0.0, prev = INFINITY;
+  while (it < adj_max_iter) {
+    idkm_ref_adjoint_apply(W, m, d, C, k, tau, S, F, u, Ju);
+    double u2 = 0.0;
+    int finite = 1;
+    averaged_step(Ju, g, u, alpha, n, un);
+    for (int t = 0; t < n; ++t) {
+      u2 += un[t] * un[t];
+      if (!isfinite(un[t])) finite = 0;
+    }
+    res = rel_change(un, u, n);
+    memcpy(u, un, sizeof(double) * (size_t)n);
+    ++it;
+    up = (res > prev) ? up + 1 : 0;
+    prev = res;
+    if (!finite || up >= 10 || sqrt(u2) > 1e6 * sqrt(g2)) {
+      diverged = 1;
+      break;
+    }
+    if (adj_tol > 0.0 && res < adj_tol) break;
+  }
+  if (iters_out) *iters_out = it;
+  if (residual_out) *residual_out = res;
+  free(Ju);
+  return diverged;
+}
+
+/* Section 4.2's safeguard as a policy: run the watched iteration with alpha0; each time it diverges start over from
+ * u = g with half the alpha, at most max_halvings times.  Returns 1 if the last attempt diverged too.  alpha_used
+ * receives the alpha of the last attempt, attempts_out the number of attempts made. */
+int idkm_ref_adjoint_solve_restart(const double *W, int64_t m, int d, const double *C, int k, double tau,
+                                   const double *S, const double *F, const double *g, double alpha0, int max_halvings,
+                                   double adj_tol, int adj_max_iter, double *u, double *alpha_used, int *attempts_out,
+                                   int *iters_out, double *residual_out) {
+  double alpha = alpha0;
+  int attempts = 0, diverged = 0;
+  for (;;) {
+    diverged = idkm_ref_adjoint_solve_watched(W, m, d, C, k, tau, S, F, g, alpha, adj_tol, adj_max_iter, u, iters_out,
+                                              residual_out);
+    ++attempts;
+    if (!diverged || attempts > max_halvings) break;
+    alpha *= 0.5;
+  }
+  if (alpha_used) *alpha_used = alpha;
+  if (attempts_out) *attempts_out = attempts;
+  return diverged;
 }
 
 /* dL/dW for L = <G, Wq>, given the adjoint u (the gradient equation dC/dW = (I - dF/dC)^-1 dF/dW at C*, contracted with g):

@@ -173,6 +173,23 @@ def adjoint_solve(W, Cm, tau: float, S, F, g, alpha: float, adj_tol: float, adj_
     return u, it.value, res.value
 
 
+def adjoint_solve_restart(W, Cm, tau: float, S, F, g, alpha0: float, max_halvings: int, adj_tol: float,
+                          adj_max_iter: int):
+    """Section 4.2's safeguard: the watched iteration, restarted with half the alpha each time it diverges.
+    Returns (u, diverged, alpha of the last attempt, attempts, iterations of the last attempt, last relative change)."""
+    W, Cm, S, F, g = _f64(W), _f64(Cm), _f64(S), _f64(F), _f64(g)
+    m, d, k = _shape(W, Cm)
+    u = np.empty((k, d))
+    it, att, res, al = C.c_int(0), C.c_int(0), C.c_double(0.0), C.c_double(0.0)
+    lib = _L()
+    lib.idkm_ref_adjoint_solve_restart.restype = C.c_int
+    div = lib.idkm_ref_adjoint_solve_restart(_p(W), C.c_int64(m), C.c_int(d), _p(Cm), C.c_int(k), C.c_double(tau), _p(S),
+                                             _p(F), _p(g), C.c_double(alpha0), C.c_int(max_halvings), C.c_double(adj_tol),
+                                             C.c_int(adj_max_iter), _p(u), C.byref(al), C.byref(att), C.byref(it),
+                                             C.byref(res))
+    return u, bool(div), al.value, att.value, it.value, res.value
+
+
 def scatter(W, G, Cm, tau: float, S, F, u) -> np.ndarray:
     W, G, Cm, S, F, u = _f64(W), _f64(G), _f64(Cm), _f64(S), _f64(F), _f64(u)
     m, d, k = _shape(W, Cm)

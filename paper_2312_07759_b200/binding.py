@@ -50,6 +50,9 @@ lib.idkm_forward_batched.argtypes = [_vp, _fp, _i64p, C.c_int, C.c_int, _fp, C.c
 lib.idkm_forward_batched.restype = C.c_int
 lib.idkm_backward.argtypes = [_vp, _fp, C.c_int, C.c_float, C.c_int, C.c_float, _fp, _fp, _vp, C.c_size_t, _vp]
 lib.idkm_backward.restype = C.c_int
+lib.idkm_backward_restart.argtypes = [_vp, _fp, C.c_float, C.c_int, C.c_float, C.c_int, _fp, _fp, _vp, C.c_size_t, _vp,
+                                      C.POINTER(C.c_float), C.POINTER(C.c_int)]
+lib.idkm_backward_restart.restype = C.c_int
 lib.idkm_get_info.argtypes = [_vp, C.POINTER(Info)]
 lib.idkm_get_info.restype = C.c_int
 lib.idkm_quantize_host.argtypes = [_vp, _fp, _i64p, C.c_int, C.c_int, _fp, C.c_int, C.c_float, C.c_float, C.c_int,
@@ -170,7 +173,8 @@ def describe_path(d: int, k: int, adj_max_iter: int = 0, adjoint_method: int = 0
     out = (C.c_int * 5)()
     _check(lib.idkm_describe_path(int(d), int(k), int(adj_max_iter), int(adjoint_method), out))
     return {"step_layout": (out[0], out[1]), "adjoint_layout": (out[2], out[3]),
-            "adjoint_route": ("fused passes", "explicit Jacobian in registers", "explicit Jacobian in tiles")[out[4]]}
+            "adjoint_route": ("fused passes", "explicit Jacobian in registers", "explicit Jacobian in tiles",
+                              "exact solve on the explicit Jacobian")[out[4]]}
 
 
 def measure_pipe_rates(stream=None):
@@ -256,6 +260,22 @@ class Context:
         _check(rc)
         return dW, dC
 
+    def backward_restart(self, dWq, adj_tol: float, adj_max_iter: int, alpha0: float = 1.0, max_halvings: int = 4, *,
+                         want_dW: bool = True, want_dC: bool = True, stream=None):
+        """``idkm_backward_restart``; returns (dW or None, dC or None, alpha of the last attempt, attempts)."""
+        import torch
+        assert dWq.is_cuda and dWq.dtype == torch.float32 and dWq.is_contiguous()
+        if self._keep is None:
+            raise IdkmError(ERR_ORDER)
+        m, d, k, L = self._shape
+        dW = torch.empty_like(dWq) if want_dW else None
+        dC = torch.empty((L * k, d), dtype=torch.float32, device=dWq.device) if want_dC else None
+        al, att = C.c_float(0.0), C.c_int(0)
+        _check(lib.idkm_backward_restart(self._h, _ptr(dWq), float(adj_tol), int(adj_max_iter), float(alpha0),
+                                         int(max_halvings), _ptr(dW), _ptr(dC), _ptr(self._ws), self._ws.numel(),
+                                         _stream(stream), C.byref(al), C.byref(att)))
+        return dW, dC, float(al.value), int(att.value)
+
     def info(self) -> List[Info]:
         arr = (Info * max(1, self.n_layers))()
         _check(lib.idkm_get_info(self._h, arr))
@@ -305,7 +325,8 @@ class Context:
         self._squared = bool(squared)
 
     def set_adjoint_method(self, method: int) -> None:
-        """0: explicit Jacobian for k*d <= 8 (default); 1: always one fused pass per adjoint step."""
+        """0: explicit Jacobian where k*d <= 64 (default); 1: always one fused pass per adjoint step; 2: exact solve
+        on the explicit Jacobian where k*d <= 64."""
         _check(lib.idkm_set_adjoint_method(self._h, int(method)))
 
     def history(self, which: int = 0, layer: int = 0, capacity: int = 1024):

@@ -521,6 +521,25 @@ static int launch_pass(idkm_ctx* ctx, int mode, PassParams* p, int repeat) {
   return IDKM_OK;
 }
 
+// The last phase of a backward: the pass that writes dL/dW from the adjoint u in the workspace, and the copy of u.
+static int backward_outputs(idkm_ctx* ctx, PassParams* p, float* dW_out, float* dC_out) {
+  if (dW_out) {
+    p->dW = dW_out;
+    nvtxRangePushA("idkm dL/dW pass");
+    const int rc = launch_pass(ctx, SCATTER, p, 1);
+    nvtxRangePop();
+    if (rc != IDKM_OK) return rc;
+  }
+  mark(ctx, 7);
+  ctx->ev_bwd_set = ctx->timing && ctx->ev_ok;
+  if (dC_out) {
+    if (cudaMemcpyAsync(dC_out, p->u, sizeof(float) * (size_t)ctx->n_layers * ctx->k * ctx->d, cudaMemcpyDeviceToDevice,
+                        ctx->stream) != cudaSuccess)
+      return IDKM_ERR_CUDA;
+  }
+  return IDKM_OK;
+}
+
 extern "C" {
 
 int idkm_create(idkm_ctx** out) {
@@ -680,7 +699,9 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   const int fj = pick_family(JACOBIAN, ctx->d, ctx->k);
   const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, ctx->d, fj)->plen > JAC_SMALL_PLEN_MAX;
   // (the explicit-Jacobian kernels are written for the Euclidean distance: the squared variant takes the fused passes)
-  const bool explicit_jac = ctx->adjoint_method == 0 && !ctx->squared && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS);
+  const bool exact = ctx->adjoint_method == 2 && !ctx->squared && fj >= 0;   // solve on the explicit matrix
+  const bool explicit_jac = exact || (ctx->adjoint_method == 0 && !ctx->squared && fj >= 0 &&
+                                      (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS));
   // the per-row softmax reference and normaliser are kept only if fused adjoint passes follow
   if (!solve || explicit_jac) p.rowstat = nullptr;
   mark(ctx, 4);
@@ -691,29 +712,52 @@ int idkm_backward(idkm_ctx* ctx, const float* dWq, idkm_mode mode, float adj_tol
   mark(ctx, 5);
   if (solve) {
     nvtxRangePushA("idkm adjoint solve");
-    if (explicit_jac)
+    if (explicit_jac) {
+      if (exact) p.max_iter = -1;                  // the epilogue solves (I - J^T) u = g instead of iterating
       rc = launch_pass(ctx, JACOBIAN, &p, 1);      // one pass forms J_C; the whole iteration runs on it in the epilogue
-    else
+      p.max_iter = adj_max_iter;
+    } else {
       rc = launch_pass(ctx, ADJ, &p, adj_max_iter);
+    }
     nvtxRangePop();
     if (rc != IDKM_OK) return rc;
   }
   mark(ctx, 6);
-  if (dW_out) {
-    p.dW = dW_out;
-    nvtxRangePushA("idkm dL/dW pass");
-    rc = launch_pass(ctx, SCATTER, &p, 1);
-    nvtxRangePop();
+  return backward_outputs(ctx, &p, dW_out, dC_out);
+}
+
+int idkm_backward_restart(idkm_ctx* ctx, const float* dWq, float adj_tol, int adj_max_iter, float alpha0,
+                          int max_halvings, float* dW_out, float* dC_out, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream, float* alpha_used_out, int* attempts_out) {
+  if (!ctx || !dWq || !workspace) return IDKM_ERR_NULL;
+  if (max_halvings < 0 || max_halvings > 30) return IDKM_ERR_PARAM;
+  if (dW_out && (!aligned16(dW_out) || dW_out == dWq || dW_out == ctx->W)) return dW_out == dWq || dW_out == ctx->W ? IDKM_ERR_PARAM : IDKM_ERR_ALIGN;
+  if (dC_out && !aligned16(dC_out)) return IDKM_ERR_ALIGN;
+  float alpha = alpha0;
+  int attempts = 0;
+  for (;;) {
+    // codebook gradient and adjoint solve only: the dL/dW pass waits for an iteration that did not diverge
+    int rc = idkm_backward(ctx, dWq, IDKM_IMPLICIT, adj_tol, adj_max_iter, alpha, nullptr, nullptr, workspace,
+                           workspace_bytes, cuda_stream);
     if (rc != IDKM_OK) return rc;
+    ++attempts;
+    idkm_info info[MAX_LAYERS];
+    rc = idkm_get_info(ctx, info);   // waits for the stream: the decision to start over is the host's
+    if (rc != IDKM_OK) return rc;
+    bool diverged = false;
+    for (int l = 0; l < ctx->n_layers; ++l) diverged = diverged || (info[l].status == IDKM_ERR_DIVERGED);
+    if (!diverged || attempts > max_halvings) break;
+    alpha *= 0.5f;
   }
-  mark(ctx, 7);
-  ctx->ev_bwd_set = ctx->timing && ctx->ev_ok;
-  if (dC_out) {
-    if (cudaMemcpyAsync(dC_out, p.u, sizeof(float) * (size_t)ctx->n_layers * ctx->k * ctx->d, cudaMemcpyDeviceToDevice,
-                        ctx->stream) != cudaSuccess)
-      return IDKM_ERR_CUDA;
-  }
-  return IDKM_OK;
+  if (alpha_used_out) *alpha_used_out = alpha;
+  if (attempts_out) *attempts_out = attempts;
+  WorkspaceLayout wl;
+  if (!make_layout(ctx->m_total, ctx->d, ctx->k, ctx->n_layers, ctx->sms, &wl)) return IDKM_ERR_UNSUPPORTED;
+  PassParams p;
+  fill_params(ctx, wl, &p);
+  p.G = dWq;
+  p.alpha = alpha;
+  return backward_outputs(ctx, &p, dW_out, dC_out);
 }
 
 int idkm_get_info(idkm_ctx* ctx, idkm_info* info_out) {
@@ -872,7 +916,7 @@ int idkm_get_phase_ms(idkm_ctx* ctx, float* ms_out) {
 
 int idkm_set_adjoint_method(idkm_ctx* ctx, int method) {
   if (!ctx) return IDKM_ERR_NULL;
-  if (method != 0 && method != 1) return IDKM_ERR_PARAM;
+  if (method < 0 || method > 2) return IDKM_ERR_PARAM;
   ctx->adjoint_method = method;
   return IDKM_OK;
 }
@@ -963,7 +1007,7 @@ int idkm_describe_path(int d, int k, int adj_max_iter, int adjoint_method, int* 
   out[3] = kernel_entry(ADJ, d, fa)->lpw;
   const bool jac_tile = fj >= 0 && kernel_entry(JACOBIAN, d, fj)->plen > JAC_SMALL_PLEN_MAX;
   const bool explicit_jac = adjoint_method == 0 && fj >= 0 && (!jac_tile || adj_max_iter >= JAC_TILE_MIN_ITERS);
-  out[4] = (adj_max_iter <= 0) ? 0 : (explicit_jac ? (jac_tile ? 2 : 1) : 0);
+  out[4] = (adj_max_iter <= 0) ? 0 : ((adjoint_method == 2 && fj >= 0) ? 3 : (explicit_jac ? (jac_tile ? 2 : 1) : 0));
   return IDKM_OK;
 }
 

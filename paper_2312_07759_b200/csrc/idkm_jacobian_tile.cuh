@@ -124,7 +124,25 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
       us[tid] = gs[tid];
     }
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 0 && p.max_iter < 0) {
+      // exact solve instead of the iteration (idkm_set_adjoint_method(ctx, 2)); gs holds g, then u
+      LayerState* st = p.st + l;
+      const bool ok = warp_solve_adjoint(Jm, KD, gs, n, lane);
+      bool finite = true;
+      for (int q = lane; q < n; q += 32) {
+        const double uv = ok ? gs[q] : 0.0;
+        finite = finite && (uv == uv) && fabs(uv) < 1e300;
+        p.u[(size_t)l * n + q] = (float)uv;
+      }
+      finite = __all_sync(0xffffffffu, finite);
+      if (lane == 0) {
+        st->ticket = 0u;
+        st->adj_iters = 0;
+        st->adj_res = 0.f;
+        st->adj_done = 1;
+        if (!ok || !finite) st->status = ST_DIVERGED;
+      }
+    } else if (warp == 0) {
       // The iteration on the matrix, by one warp: lane q owns coordinates q and q + 32 of u;
       // (J^T u)_q = sum_r J[r][q] u_r with J and u in shared memory.  All lanes see the same residual.
       LayerState* st = p.st + l;

@@ -1361,6 +1361,81 @@ idkm_step_dual(const __grid_constant__ DualParams dp) {
 }
 
 
+// Exact solve of (I - J^T) u = g -- the linear system behind M* = (I - dF/dC)^-1 of Section 4.2, contracted with g --
+// by ONE warp: the matrix J (n x n, row stride ld, fp64, shared memory) is turned into I - J^T in place, then Gaussian
+// elimination with partial pivoting and back substitution.  b holds g on entry and u on exit.  Lanes take columns
+// (consecutive addresses: no bank conflicts), rows run in a loop.  Returns false when a pivot vanishes or is not a
+// number (J has an eigenvalue 1 to working precision, or the sums were not finite).  n <= 64.
+__device__ __forceinline__ bool warp_solve_adjoint(double* J, int ld, double* b, int n, int lane) {
+  for (int idx = lane; idx < n * n; idx += 32) {
+    const int r = idx / n, c = idx % n;
+    if (r < c) {
+      const double x = J[r * ld + c], y = J[c * ld + r];
+      J[r * ld + c] = -y;
+      J[c * ld + r] = -x;
+    } else if (r == c) {
+      J[r * ld + r] = 1.0 - J[r * ld + r];
+    }
+  }
+  __syncwarp();
+  bool ok = true;
+  for (int c = 0; c < n; ++c) {
+    double best = -1.0;
+    int br = c;
+    for (int r = c + lane; r < n; r += 32) {
+      const double v = fabs(J[r * ld + c]);
+      if (v > best) {
+        best = v;
+        br = r;
+      }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int orow = __shfl_xor_sync(0xffffffffu, br, o);
+      if (ob > best || (ob == best && orow < br)) {
+        best = ob;
+        br = orow;
+      }
+    }
+    if (!(best > 0.0) || !(best < 1e300)) {
+      ok = false;
+      break;
+    }
+    if (br != c) {
+      for (int q = lane; q < n; q += 32) {
+        const double x = J[c * ld + q];
+        J[c * ld + q] = J[br * ld + q];
+        J[br * ld + q] = x;
+      }
+      if (lane == 0) {
+        const double x = b[c];
+        b[c] = b[br];
+        b[br] = x;
+      }
+    }
+    __syncwarp();
+    const double inv_piv = 1.0 / J[c * ld + c];
+    const double bc = b[c];
+    for (int r = c + 1; r < n; ++r) {
+      const double f = J[r * ld + c] * inv_piv;
+      for (int q = c + 1 + lane; q < n; q += 32) J[r * ld + q] = fma(-f, J[c * ld + q], J[r * ld + q]);
+      if (lane == 0) b[r] = fma(-f, bc, b[r]);
+    }
+    __syncwarp();
+  }
+  if (!ok) return false;
+  for (int r = n - 1; r >= 0; --r) {
+    double sres = 0.0;
+    for (int q = r + 1 + lane; q < n; q += 32) sres = fma(J[r * ld + q], b[q], sres);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sres += __shfl_xor_sync(0xffffffffu, sres, o);
+    if (lane == 0) b[r] = (b[r] - sres) / J[r * ld + r];
+    __syncwarp();
+  }
+  return true;
+}
+
 // ---- explicit Jacobian for small codebooks -------------------------------------------------------------------
 // When k d <= 8 the matrix J_C = dF/dC (k d x k d, at most 64 entries) fits in a thread's registers.  One pass over
 // W accumulates it -- J[(j,a),(l,b)] = sum_i P_ija (delta_jl - A_il) n_ilb with P_ija = A_ij (w_ia - F_ja) / (S_j tau)
@@ -1456,7 +1531,28 @@ __global__ void __launch_bounds__(BLOCK) idkm_jacobian(const __grid_constant__ P
       }
       __syncthreads();
     }
-    if (warp == 0) {
+    if (warp == 0 && p.max_iter < 0) {
+      // exact solve instead of the iteration (idkm_set_adjoint_method(ctx, 2))
+      LayerState* st = p.st + l;
+      const int n = k * D;
+      if (lane < n) scratch[lane] = (double)p.gvec[(size_t)l * n + lane];
+      __syncwarp();
+      const bool ok = warp_solve_adjoint(tot, KD, scratch, n, lane);
+      bool finite = true;
+      if (lane < n) {
+        const double uv = ok ? scratch[lane] : 0.0;
+        finite = (uv == uv) && fabs(uv) < 1e300;
+        p.u[(size_t)l * n + lane] = (float)uv;
+      }
+      finite = __all_sync(0xffffffffu, finite);
+      if (lane == 0) {
+        st->ticket = 0u;
+        st->adj_iters = 0;
+        st->adj_res = 0.f;
+        st->adj_done = 1;
+        if (!ok || !finite) st->status = ST_DIVERGED;
+      }
+    } else if (warp == 0) {
       // The iteration on the small matrix, by one warp: lane q < n owns coordinate q of u and column q of J
       // (J^T u)_q = sum_r J[r][q] u_r; u_r is fetched from lane r by a shuffle.  All lanes see the same residual.
       LayerState* st = p.st + l;
