@@ -219,6 +219,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=1 << 19, help="rows of the workload the oracle is timed on")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--collapse-step", type=int, default=0, choices=[0, 1],
+                    help="step of collapsing layers: 0 fp32 increment form (default), 1 fp64")
     ap.add_argument("--iters", type=int, default=0, help="override the forward and adjoint iteration counts "
                     "(short runs for profiler captures; the reported value is then not the configured workload's)")
     args = ap.parse_args()
@@ -252,6 +254,7 @@ def main():
     C0 = torch.from_numpy(wl.C0).to(dev)
     G = torch.from_numpy(wl.G).to(dev)
     ctx = B.Context()
+    ctx.set_collapse_step(args.collapse_step)
     ctx.set_timing(True)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)     # > 126 MB L2
 

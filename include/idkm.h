@@ -324,6 +324,19 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 
 /*
+ * How the forward step treats a COLLAPSING layer, i.e. one whose centroids all lie within 0.0625 tau of each other
+ * (tau above the spread of the weights: every centroid slides into the mean).  There the update of C is decided by
+ * attention differences far below fp32 resolution of w - c_j, so such layers leave the ordinary fp32 step.
+ * 0 (default): an fp32 step in the increment form -- with u_i = w_i - c_0 and delta_j = c_j - c_0 the logit
+ * differences -(D_ij - D_i0) / tau, the attention increments A_ij - 1/k and the sums of (A_ij - 1/k) and
+ * (A_ij - 1/k) u_i are all small quantities evaluated to fp32 relative accuracy; the M-step is completed in fp64 from
+ * those sums and sum_i u_i.  1: the same step with fp64 distances, exponentials and sums (about four times slower per
+ * row; kept as the reference for the other).  Both realise Algorithm 1's steps 3-5 for such layers and agree with
+ * the float64 oracle within the stated tolerance.  Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_PARAM.
+ */
+int idkm_set_collapse_step(idkm_ctx* ctx, int method);
+
+/*
  * Host-side fault injection for tests of the timeout path of the one-launch forward loop (no GPU fault is involved:
  * the waits stay bounded and the kernel returns).  missing_arrivals = n > 0 makes each grid-wide barrier of this
  * ctx's following calls wait for n arrivals that never come; spin_limit_ticks > 0 shortens the bound of every wait

@@ -74,6 +74,8 @@ lib.idkm_set_test_hooks.argtypes = [_vp, C.c_int, C.c_int64]
 lib.idkm_set_test_hooks.restype = C.c_int
 lib.idkm_count_busy_tickets.argtypes = [_vp, C.POINTER(C.c_int)]
 lib.idkm_count_busy_tickets.restype = C.c_int
+lib.idkm_set_collapse_step.argtypes = [_vp, C.c_int]
+lib.idkm_set_collapse_step.restype = C.c_int
 lib.idkm_set_distance.argtypes = [_vp, C.c_int]
 lib.idkm_set_distance.restype = C.c_int
 lib.idkm_set_adjoint_method.argtypes = [_vp, C.c_int]
@@ -317,6 +319,10 @@ class Context:
         _check(rc)
         self.n_layers = L
         return Cout, Wq, dW, dC, list(infos)
+
+    def set_collapse_step(self, method: int) -> None:
+        """``idkm_set_collapse_step``: 0 = collapsing layers step in the fp32 increment form (default), 1 = in fp64."""
+        _check(lib.idkm_set_collapse_step(self._h, int(method)))
 
     def set_distance(self, squared: bool) -> None:
         """``idkm_set_distance``: False = Euclidean distance in the softmax (Algorithm 1), True = its square."""

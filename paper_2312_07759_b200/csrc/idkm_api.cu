@@ -29,6 +29,8 @@ extern const KernelEntry k_table_step_precise[3][N_FAMILY];
 extern const KernelEntry k_table_jacobian[3][N_FAMILY];
 extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY];
 extern const DualEntry k_table_dual[3][2];
+extern const DualEntry k_table_dual_delta[3][2];
+extern const KernelEntry k_table_step_delta[3][N_FAMILY];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
@@ -89,6 +91,7 @@ const KernelEntry* kernel_entry(int mode, int d, int family) {
     case ADJ: return &k_table_adj[di][family];
     case SCATTER: return &k_table_scatter[di][family];
     case STEP_PRECISE: return &k_table_step_precise[di][family];
+    case STEP_DELTA: return &k_table_step_delta[di][family];
     case JACOBIAN: return &k_table_jacobian[di][family];
   }
   return nullptr;
@@ -122,11 +125,14 @@ int pick_family(int mode, int d, int k) {
   // forward step with more than 128 centroids: for d <= 2 the 8-centroids-per-lane, full-warp layout at two blocks
   // per SM is faster than 16 centroids per lane on half-warps (m = 2^22, k = 256: d = 1 0.46 against 0.54 ms, d = 2
   // 0.71 against 0.77 ms); for d = 4 the half-warp layout wins (0.90 against 0.95 ms)
-  if (mode == STEP && k > 128 && d < 4) return N_FAMILY - 1;
+  if (mode == STEP && k > 128 && d < 4) return FAM_WIDE;
   // adjoint step with more than 128 centroids at d = 4: 16 centroids per lane on half-warps (m = 2^22, k = 256:
   // 1.22 against 1.29 ms for 8 per lane on full warps)
-  if (mode == ADJ && k > 128 && d == 4) return N_FAMILY - 1;
-  for (int f = 0; f < N_FAMILY; ++f) {
+  if (mode == ADJ && k > 128 && d == 4) return FAM_WIDE;
+  // forward step with 9..16 centroids at d >= 2: 8 centroids per lane on lane pairs at two blocks per SM instead of 16
+  // per thread at one (m = 2^24, k = 16: d = 4 0.28 against 0.50 ms, d = 2 0.19 against 0.22 ms; d = 1 0.13 against 0.12)
+  if (mode == STEP && k > 8 && k <= 16 && d >= 2) return FAM_8x2;
+  for (int f = 0; f <= FAM_WIDE; ++f) {
     const KernelEntry* e = kernel_entry(mode, d, f);
     if (e && e->launch && e->kpl * e->lpw >= k) return f;
   }
@@ -144,11 +150,11 @@ constexpr int JAC_TILE_MIN_ITERS = 16;
 
 // The dual step kernel of (d, k), or null: it exists for the layouts (2,1) and (4,1) where the fp32 and the fp64 step
 // pick the same layout and register budget.
-static const DualEntry* dual_entry(int d, int k) {
+static const DualEntry* dual_entry(int d, int k, bool delta = true) {
   const int di = d == 1 ? 0 : (d == 2 ? 1 : (d == 4 ? 2 : -1));
   const int f = pick_family(STEP, d, k);
-  if (di < 0 || f < 0 || f > 1 || pick_family(STEP_PRECISE, d, k) != f) return nullptr;
-  const DualEntry* e = &k_table_dual[di][f];
+  if (di < 0 || f < 0 || f > 1 || pick_family(STEP_PRECISE, d, k) != f || pick_family(STEP_DELTA, d, k) != f) return nullptr;
+  const DualEntry* e = delta ? &k_table_dual_delta[di][f] : &k_table_dual[di][f];
   return e->launch ? e : nullptr;
 }
 
@@ -205,7 +211,8 @@ static bool make_layout(int64_t m_total, int d, int k, int n_layers, int sms, Wo
   w.off_hist_fwd = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
   w.off_hist_adj = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
   const DualEntry* de = dual_entry(d, k);
-  const int plen64 = de ? kernel_entry(STEP_PRECISE, d, pick_family(STEP_PRECISE, d, k))->plen : 0;
+  // (the second half of the dual kernel is the fp64 step or the fp32 increment-form step: room for the larger partial)
+  const int plen64 = de ? kernel_entry(STEP_DELTA, d, pick_family(STEP_DELTA, d, k))->plen : 0;
   w.max_groups64 = de ? w.max_groups : 0;
   w.off_partials64 = o;  o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen64, 256);
   w.off_gpartials64 = o; o = align_up(o + sizeof(double) * (size_t)w.max_groups64 * plen64, 256);
@@ -259,6 +266,7 @@ struct idkm_ctx {
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
   int squared;          // 1: squared-distance variant (idkm_set_distance)
+  int collapse_step;    // 0: collapsing layers step in the fp32 increment form; 1: in fp64 (idkm_set_collapse_step)
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
   int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never;
                         // 2: never, and the fp32 and fp64 steps of an iteration are always two launches
@@ -329,7 +337,7 @@ static int build_table(idkm_ctx* ctx, int mode, int family, LayerTable* lt) {
   // and the blocks that own their tiles return at once.  With more blocks than fit on the GPU at a time the
   // hardware scheduler backfills the freed slots with blocks of the layers that still run, instead of leaving SMs
   // idle for the rest of the launch.
-  if (ctx->n_layers > 1 && (mode == STEP || mode == STEP_PRECISE || mode == ADJ)) nb = (long long)ctx->sms * MAX_BLOCKS_PER_SM;
+  if (ctx->n_layers > 1 && (mode == STEP || mode == STEP_PRECISE || mode == STEP_DELTA || mode == ADJ)) nb = (long long)ctx->sms * MAX_BLOCKS_PER_SM;
   if (nb > tiles) nb = tiles;
   lt->n_blocks = (int)nb;
   lt->pad = 0;
@@ -396,15 +404,18 @@ struct RunAhead {
 // The forward loop: every iteration launches the fp32 step and the fp64 step; each layer is taken by exactly one
 // of them (LayerState::precise), the other returns at once for it.
 static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p, int repeat) {
-  const int f32 = pick_family(STEP, ctx->d, ctx->k), f64 = pick_family(STEP_PRECISE, ctx->d, ctx->k);
+  // the step of the collapsing layers: fp32 in the increment form, or fp64
+  const int mode64 = ctx->collapse_step == 0 ? STEP_DELTA : STEP_PRECISE;
+  const int f32 = pick_family(STEP, ctx->d, ctx->k), f64 = pick_family(mode64, ctx->d, ctx->k);
   const KernelEntry* e32 = ctx_entry(ctx, STEP, f32);
-  const KernelEntry* e64 = kernel_entry(STEP_PRECISE, ctx->d, f64);
+  const KernelEntry* e64 = kernel_entry(mode64, ctx->d, f64);
   static const bool dual_off = (getenv("IDKM_NO_DUAL") != nullptr);   // tuning knob: always two launches per iteration
-  const DualEntry* de = (dual_off || ctx->forward_loop == 2 || ctx->squared) ? nullptr : dual_entry(ctx->d, ctx->k);
+  const DualEntry* de = (dual_off || ctx->forward_loop == 2 || ctx->squared) ? nullptr
+                                                                             : dual_entry(ctx->d, ctx->k, mode64 == STEP_DELTA);
   PassParams q = *p;
   int rc = build_table(ctx, STEP, f32, &p->lt);
   if (rc != IDKM_OK) return rc;
-  rc = build_table(ctx, STEP_PRECISE, f64, &q.lt);
+  rc = build_table(ctx, mode64, f64, &q.lt);
   if (rc != IDKM_OK) return rc;
   int dual_grid = 0;
   if (de) {
@@ -948,6 +959,13 @@ int idkm_set_distance(idkm_ctx* ctx, int squared) {
   if (squared != 0 && squared != 1) return IDKM_ERR_PARAM;
   if (ctx->squared != squared) ctx->have_forward = false;   // a backward must follow a forward of the same variant
   ctx->squared = squared;
+  return IDKM_OK;
+}
+
+int idkm_set_collapse_step(idkm_ctx* ctx, int method) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (method != 0 && method != 1) return IDKM_ERR_PARAM;
+  ctx->collapse_step = method;
   return IDKM_OK;
 }
 

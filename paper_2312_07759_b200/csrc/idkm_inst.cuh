@@ -66,7 +66,8 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
   {                                                                                               \
     IDKM_PRECISE_ENTRY(D, 2, 1), IDKM_PRECISE_ENTRY(D, 4, 1), IDKM_PRECISE_ENTRY(D, 8, 1),        \
         IDKM_PRECISE_ENTRY(D, 8, 2), IDKM_PRECISE_ENTRY(D, 8, 4), IDKM_PRECISE_ENTRY(D, 8, 8),    \
-        IDKM_PRECISE_ENTRY(D, 8, 16), IDKM_PRECISE_ENTRY(D, 8, 32), IDKM_PRECISE_ENTRY(D, 8, 32)  \
+        IDKM_PRECISE_ENTRY(D, 8, 16), IDKM_PRECISE_ENTRY(D, 8, 32), IDKM_PRECISE_ENTRY(D, 8, 32), \
+        IDKM_NO_ENTRY, IDKM_NO_ENTRY                                                              \
   }
 
 template <int D, int KPL>
@@ -85,13 +86,15 @@ static cudaError_t launch_jacobian(const PassParams& p, int grid, cudaStream_t s
   {                                                                                               \
     IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
         IDKM_ENTRY(MODE, D, 16, 1), IDKM_ENTRY(MODE, D, 16, 2), IDKM_ENTRY(MODE, D, 16, 4),       \
-        IDKM_ENTRY(MODE, D, 16, 8), IDKM_ENTRY(MODE, D, 16, 16), IDKM_ENTRY(MODE, D, 8, 32)       \
+        IDKM_ENTRY(MODE, D, 16, 8), IDKM_ENTRY(MODE, D, 16, 16), IDKM_ENTRY(MODE, D, 8, 32),      \
+        IDKM_ENTRY(MODE, D, 4, 4), IDKM_ENTRY(MODE, D, 8, 2)                                      \
   }
 #define IDKM_BWD_ROW(MODE, D)                                                                     \
   {                                                                                               \
     IDKM_ENTRY(MODE, D, 2, 1), IDKM_ENTRY(MODE, D, 4, 1), IDKM_ENTRY(MODE, D, 8, 1),              \
         IDKM_ENTRY(MODE, D, 8, 2), IDKM_ENTRY(MODE, D, 8, 4), IDKM_ENTRY(MODE, D, 8, 8),          \
-        IDKM_ENTRY(MODE, D, 8, 16), IDKM_ENTRY(MODE, D, 8, 32), IDKM_ENTRY(MODE, D, 8, 32)        \
+        IDKM_ENTRY(MODE, D, 8, 16), IDKM_ENTRY(MODE, D, 8, 32), IDKM_ENTRY(MODE, D, 8, 32),       \
+        IDKM_ENTRY(MODE, D, 4, 4), IDKM_ENTRY(MODE, D, 8, 2)                                      \
   }
 // The adjoint step's last entry is the half-warp layout with 16 centroids per lane (one block of 8 warps per SM,
 // 254 registers): half the per-row overhead and one shuffle stage fewer per pair than 8 centroids on a full warp, and
@@ -100,7 +103,8 @@ static cudaError_t launch_jacobian(const PassParams& p, int grid, cudaStream_t s
   {                                                                                               \
     IDKM_ENTRY(ADJ, D, 2, 1), IDKM_ENTRY(ADJ, D, 4, 1), IDKM_ENTRY(ADJ, D, 8, 1),                 \
         IDKM_ENTRY(ADJ, D, 8, 2), IDKM_ENTRY(ADJ, D, 8, 4), IDKM_ENTRY(ADJ, D, 8, 8),             \
-        IDKM_ENTRY(ADJ, D, 8, 16), IDKM_ENTRY(ADJ, D, 8, 32), IDKM_ENTRY(ADJ, D, 16, 16)          \
+        IDKM_ENTRY(ADJ, D, 8, 16), IDKM_ENTRY(ADJ, D, 8, 32), IDKM_ENTRY(ADJ, D, 16, 16),         \
+        IDKM_ENTRY(ADJ, D, 4, 4), IDKM_ENTRY(ADJ, D, 8, 2)                                        \
   }
 
 }  // namespace idkm

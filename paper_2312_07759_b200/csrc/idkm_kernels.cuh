@@ -41,8 +41,8 @@ constexpr double PRECISE_SPAN = 0.0625;
 // as well; a spiralling (complex-eigenvalue) divergence shows only in the norm.
 constexpr double ADJ_GROWTH_LIMIT = 1e6;
 
-enum Mode { STEP = 0, FINAL = 1, GRAD = 2, ADJ = 3, SCATTER = 4, STEP_PRECISE = 5, JACOBIAN = 6 };
-constexpr int N_MODES = 7;
+enum Mode { STEP = 0, FINAL = 1, GRAD = 2, ADJ = 3, SCATTER = 4, STEP_PRECISE = 5, JACOBIAN = 6, STEP_DELTA = 7 };
+constexpr int N_MODES = 8;
 
 // status values mirrored from idkm.h (device side needs only these)
 constexpr int ST_OK = 0, ST_MAXITER = 1, ST_NONFINITE = -9, ST_DIVERGED = -10, ST_TIMEOUT = -12;
@@ -136,8 +136,12 @@ struct PassCfg {
   // resident blocks per SM the register budget is sized for (the 32-lane layouts hold 8 centroids per lane)
   // (thread-per-weight: estimated from the registers that hold centroids, per-centroid constants and sums)
   static constexpr int REGS_EST = KPL * ((MODE == STEP || MODE == FINAL) ? 2 * D + 1 : 3 * D + 1) + 40;
+  // (the two 16-centroid group layouts: three resp. two blocks, their centroids and sums need 36 resp. 72 registers)
   static constexpr int MIN_BLOCKS =
-      (LPW == 32) ? 2 : ((LPW > 1) ? 1 : ((256 / REGS_EST) > 4 ? 4 : ((256 / REGS_EST) < 1 ? 1 : (256 / REGS_EST))));
+      (LPW == 32) ? 2
+      : (KPL == 4 && LPW == 4) ? 3
+      : (KPL == 8 && LPW == 2 && (MODE == STEP || MODE == FINAL)) ? 2
+      : ((LPW > 1) ? 1 : ((256 / REGS_EST) > 4 ? 4 : ((256 / REGS_EST) < 1 ? 1 : (256 / REGS_EST))));
 };
 
 // Layouts whose adjoint step reads each row's softmax reference and normaliser from the workspace instead of
@@ -249,7 +253,10 @@ __device__ __forceinline__ double block_sum_double(double v, double* scratch) { 
 // pass.  Grouping and order depend on block indices only, so the result is reproducible.  Layers with at most
 // RED_SINGLE_MAX contributing blocks skip the first stage.  Called by all threads of the block.
 // smem_raw must hold (PLEN + BLOCK) doubles.
-template <int MODE, int D, int PLEN, int NA>
+// DELTA (forward step of a collapsing layer in the increment form, see delta_body): the totals are
+// dS_j = sum_i (A_ij - 1/k), dN_j = sum_i (A_ij - 1/k) (w_i - c_0) and, in the last D entries, sum_i w_i; with
+// U = sum_i w_i - m c_0 the M-step is C+_j = c_0 + (U / k + dN_j) / (m / k + dS_j).
+template <int MODE, int D, int PLEN, int NA, bool DELTA = false>
 __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, unsigned char* smem_raw, int* s_flag) {
   const int tid = threadIdx.x;
   const int k = p.k;
@@ -337,15 +344,53 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   }
   if constexpr (MODE == STEP) {
     float* Cl = p.C + (size_t)l * k * D;
+    double c0[D], ubar[D], mk = 0.0;
+    (void)c0; (void)ubar; (void)mk;
+    if constexpr (DELTA) {
+      constexpr int NEXTRA = (D == 1) ? 4 : 0;
+      const double mrows = (double)(p.lt.row_off[l + 1] - p.lt.row_off[l]);
+      mk = mrows / (double)k;
+      double wsum[D];
+#pragma unroll
+      for (int a = 0; a < D; ++a) {
+        c0[a] = (double)Cl[a];                       // centroid 0 before anybody overwrites it
+        wsum[a] = tot[PLEN - NEXTRA - D + a];
+      }
+      if constexpr (D == 1) {
+        // Scalar weights outside the centroids see the logits +-delta_j / tau, whatever their own value: their
+        // attention increments take two values per centroid, a+_j for w > c and a-_j for w < c, and the row loop only
+        // counted them (cp, cm) and added their weights up (sp, sm).  Their share of dS_j and dN_j is added here.
+        const double cp = tot[PLEN - 4], sp = tot[PLEN - 3], cm = tot[PLEN - 2], sm = tot[PLEN - 1];
+        wsum[0] += sp + sm;
+        // (k <= BLOCK: one centroid per thread; fixed-order block sums for the two means)
+        double tpj = 0.0, tmj = 0.0;
+        if (tid < k) {
+          const double dj = ((double)Cl[tid] - c0[0]) * p.inv_tau_d;
+          tpj = expm1(dj);
+          tmj = expm1(-dj);
+        }
+        const double tbp = block_sum_double(tpj, scratch) / (double)k;
+        const double tbm = block_sum_double(tmj, scratch) / (double)k;
+        if (tid < k) {
+          const double ap = (tpj - tbp) / ((double)k * (1.0 + tbp));
+          const double am = (tmj - tbm) / ((double)k * (1.0 + tbm));
+          tot[tid * NA] += ap * cp + am * cm;
+          tot[tid * NA + 1] += ap * (sp - cp * c0[0]) + am * (sm - cm * c0[0]);
+        }
+      }
+#pragma unroll
+      for (int a = 0; a < D; ++a) ubar[a] = (wsum[a] - mrows * c0[a]) / (double)k;
+      __syncthreads();
+    }
     for (int j = tid; j < k; j += BLOCK) {
-      const double s = tot[j * NA];
+      const double s = DELTA ? mk + tot[j * NA] : tot[j * NA];
       const bool alive = (s >= S_MIN);
       if (!alive) dead += 1.0;
       if (!(s == s) || s > 1e300) bad += 1.0;
 #pragma unroll
       for (int a = 0; a < D; ++a) {
         const double cold = (double)Cl[j * D + a];
-        const double cnew = alive ? tot[j * NA + 1 + a] / s : cold;
+        const double cnew = alive ? (DELTA ? c0[a] + (ubar[a] + tot[j * NA + 1 + a]) / s : tot[j * NA + 1 + a] / s) : cold;
         if (!(cnew == cnew) || fabs(cnew) > 1e300) bad += 1.0;
         num += (cnew - cold) * (cnew - cold);
         den += cnew * cnew;
@@ -1342,6 +1387,368 @@ idkm_step_precise(const __grid_constant__ PassParams p) {
   precise_body<D, KPL, LPW>(p);
 }
 
+// ---- fp32 forward step for collapsing layers in the increment form ---------------------------------------------
+// The same M-step as the STEP pass for the layers flagged `precise`, without fp64 in the row loop.  In such a layer
+// every centroid lies within PRECISE_SPAN * tau of centroid 0, so with u_i = w_i - c_0 and delta_j = c_j - c_0
+// (formed in fp64, rounded once):
+//   D_ij^2 - D_i0^2 = |delta_j|^2 - 2 delta_j . u_i =: q_ij,      D_ij - D_i0 = q_ij / (D_ij + D_i0)
+//   (d = 1: D_ij - D_i0 = |u_i - delta_j| - |u_i| = -sign(u_i) delta_j for every weight outside [c_0, c_j])
+//   x_ij = -(D_ij - D_i0) / tau,  |x_ij| <= PRECISE_SPAN,   t_ij = exp(x_ij) - 1 by a fifth-degree series,
+//   A_ij - 1/k = (t_ij - tbar_i) / (k (1 + tbar_i)),   tbar_i = mean_j t_ij.
+// Every quantity is small and known to fp32 RELATIVE accuracy -- errors scale with delta, not with |w| -- which is
+// what the fp32 STEP pass loses (its w - c_j rounds on the grid of w).  Accumulated per centroid:
+// dS_j = sum_i (A_ij - 1/k) and dN_j = sum_i (A_ij - 1/k) u_i, and once per layer sum_i w_i (of the weights themselves:
+// the fp32 difference w_i - c_0 rounds the same way for every weight of a binade, harmless relative to u_i in dN_j but a
+// bias in a plain sum; U = sum_i w_i - m c_0 is formed in fp64); the epilogue forms
+// C+_j = c_0 + (U / k + dN_j) / (m / k + dS_j) in fp64 (finish_layer with DELTA).  Sums are two-level like the STEP
+// pass (fp32 per about 64 rows, then a private shared-memory slot; fp64 across blocks).
+template <int D, int KPL, int LPW>
+struct DeltaCfg {
+  static constexpr int KP = KPL * LPW;
+  static constexpr int NA = D + 1;
+  static constexpr int PLENK = KP * NA;
+  // after the per-centroid sums: D entries for the sum of the weights and, for scalar weights, the four sums of the
+  // rows that need no per-centroid work (see delta_body)
+  static constexpr int NEXTRA = (D == 1) ? 4 : 0;
+  static constexpr int PLEN = PLENK + D + NEXTRA;
+  static constexpr int VEC = 4 / D;                  // rows per 128-bit load (thread-per-weight layouts)
+  static constexpr int UN = 4;                       // 128-bit loads in flight per thread and trip
+  static constexpr int WPG = (LPW == 1) ? VEC * UN : 16;   // rows per thread (per group) and tile
+  static constexpr int TILE = (BLOCK / LPW) * WPG;
+  static constexpr int NSLOT = KPL * NA + D + NEXTRA;   // second-level sums per thread
+  static constexpr int DYN_SMEM = BLOCK * NSLOT * 4;
+  static constexpr int SPILL_TILES = (64 / WPG) > 0 ? (64 / WPG) : 1;
+  static constexpr int MIN_BLOCKS = (LPW == 1 && KPL * NA <= 8) ? 4 : ((KPL * NA <= 24) ? 2 : 1);
+};
+
+// exp(x) - 1 for |x| <= PRECISE_SPAN: x + x^2 (1/2 + x (1/6 + x (1/24 + x/120))), truncation x^5 / 720 < 2e-9
+// relative; five instructions
+__device__ __forceinline__ float expm1_small(float x) {
+  float s = fmaf(x, 1.f / 120.f, 1.f / 24.f);
+  s = fmaf(s, x, 1.f / 6.f);
+  s = fmaf(s, x, 0.5f);
+  return fmaf(s * x, x, x);
+}
+
+template <int D, int KPL, int LPW>
+__device__ __forceinline__ void delta_body(const PassParams& p) {
+  using Cfg = DeltaCfg<D, KPL, LPW>;
+  constexpr int NA = Cfg::NA, PLEN = Cfg::PLEN, PLENK = Cfg::PLENK, WPG = Cfg::WPG, TILE = Cfg::TILE, NSLOT = Cfg::NSLOT;
+  constexpr int NEXTRA = Cfg::NEXTRA;
+  constexpr int RED_BYTES = NWARP * PLEN * 4;
+  constexpr int LAST_BYTES = (PLEN + BLOCK) * 8;
+  constexpr int SMEM_BYTES = RED_BYTES > LAST_BYTES ? RED_BYTES : LAST_BYTES;
+  __shared__ __align__(16) unsigned char smem_raw[SMEM_BYTES];
+  __shared__ int s_flag;
+  extern __shared__ __align__(16) float slots[];   // [NSLOT][BLOCK]
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int gl = (LPW == 1) ? 0 : (lane % LPW);
+  const int grp = tid / LPW;
+  const int k = p.k;
+  const int nb = p.lt.n_blocks;
+  const int b = blockIdx.x;
+  const int t_lo = tile_begin(b, p.lt.tiles_total, nb);
+  const int t_hi = tile_begin(b + 1, p.lt.tiles_total, nb);
+  if (b >= nb || t_lo >= t_hi) return;
+
+  float dl[KPL][D], dl2[KPL], c0[D];
+  float acc[KPL][NA], uacc[D];
+  // scalar weights: count and sum of the rows above / below all centroids (cp, sp, cm, sm), which need no
+  // per-centroid work (their attention increments take two values per centroid, applied in the epilogue)
+  float fx[NEXTRA > 0 ? NEXTRA : 1];
+  float dmax2 = 0.f;      // twice the largest |delta_j|: rows farther than this from c_0 are outside the centroids
+  (void)fx; (void)dmax2;
+  bool cvalid[KPL];
+  float inv_k = 0.f;
+  int layer = 0;
+  while (p.lt.tile_off[layer + 1] <= t_lo) ++layer;
+  int cur_layer = -1;
+  bool layer_active = false;
+  int since_spill = 0;
+
+  auto spill = [&]() {
+#pragma unroll
+    for (int t = 0; t < KPL; ++t)
+#pragma unroll
+      for (int a = 0; a < NA; ++a) {
+        slots[(t * NA + a) * BLOCK + tid] += acc[t][a];
+        acc[t][a] = 0.f;
+      }
+#pragma unroll
+    for (int a = 0; a < D; ++a) {
+      slots[(KPL * NA + a) * BLOCK + tid] += uacc[a];
+      uacc[a] = 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < NEXTRA; ++q) {
+      slots[(KPL * NA + D + q) * BLOCK + tid] += fx[q];
+      fx[q] = 0.f;
+    }
+  };
+
+  auto flush = [&](int l) {
+    float* red = reinterpret_cast<float*>(smem_raw);   // [NWARP][PLEN]
+    // per-centroid sums: across the groups of a warp (lanes with equal gl); U: once per group (its lanes hold copies)
+#pragma unroll
+    for (int t = 0; t < KPL; ++t)
+#pragma unroll
+      for (int a = 0; a < NA; ++a) {
+        float v = acc[t][a] + slots[(t * NA + a) * BLOCK + tid];
+#pragma unroll
+        for (int o = LPW; o < 32; o <<= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        acc[t][a] = v;
+      }
+#pragma unroll
+    for (int a = 0; a < D; ++a) {
+      float v = (gl == 0) ? uacc[a] + slots[(KPL * NA + a) * BLOCK + tid] : 0.f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      uacc[a] = v;
+    }
+    __syncthreads();
+    if (lane < LPW) {
+#pragma unroll
+      for (int t = 0; t < KPL; ++t)
+#pragma unroll
+        for (int a = 0; a < NA; ++a) red[warp * PLEN + (gl * KPL + t) * NA + a] = acc[t][a];
+    }
+    float fxs[NEXTRA > 0 ? NEXTRA : 1];
+    (void)fxs;
+#pragma unroll
+    for (int q = 0; q < NEXTRA; ++q) {
+      float v = (gl == 0) ? fx[q] + slots[(KPL * NA + D + q) * BLOCK + tid] : 0.f;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      fxs[q] = v;
+    }
+    if (lane == 0) {
+#pragma unroll
+      for (int a = 0; a < D; ++a) red[warp * PLEN + PLENK + a] = uacc[a];
+#pragma unroll
+      for (int q = 0; q < NEXTRA; ++q) red[warp * PLEN + PLENK + D + q] = fxs[q];
+    }
+    __syncthreads();
+    double* mine = p.partials + (size_t)(b + l) * PLEN;
+    for (int o = tid; o < PLEN; o += BLOCK) {
+      double sres = 0.0;
+#pragma unroll
+      for (int wv = 0; wv < NWARP; ++wv) sres += (double)red[wv * PLEN + o];
+      mine[o] = sres;
+    }
+    finish_layer<STEP, D, PLEN, NA, true>(p, l, b, smem_raw, &s_flag);
+  };
+
+  // full_tag: the codebook fills every centroid slot of the layout (no per-centroid validity tests)
+  auto row = [&](const float (&w)[D], bool ok, auto full_tag) {
+    constexpr bool FULL = decltype(full_tag)::value;
+    float u[D];
+#pragma unroll
+    for (int a = 0; a < D; ++a) u[a] = w[a] - c0[a];
+    float x[KPL];
+    if constexpr (D == 1) {
+      // |u - delta| - |u| without forming u - delta (which would round delta on the grid of u): -sign(u) delta when
+      // c_0 and c_j lie on the same side of the weight, |delta| - 2 |u| when the weight lies between them
+      // (with s = sign(u): -s delta + 2 max(0, s delta - |u|), branch-free)
+      const float u0 = u[0], aut = fabsf(u0) * p.inv_tau;
+      const float sg = copysignf(p.inv_tau, u0);           // s / tau
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        const float sd = sg * dl[t][0];                     // s delta / tau
+        x[t] = fmaf(-2.f, fmaxf(sd - aut, 0.f), sd);        // -(D_ij - D_i0) / tau
+      }
+    } else {
+      float d0sq = 0.f;
+#pragma unroll
+      for (int a = 0; a < D; ++a) d0sq = fmaf(u[a], u[a], d0sq);
+      const float d0 = sqrt_approx(d0sq);
+      float v[D];
+#pragma unroll
+      for (int a = 0; a < D; ++a) v[a] = -2.f * u[a];
+#pragma unroll
+      for (int t = 0; t < KPL; ++t) {
+        float q = dl2[t];
+#pragma unroll
+        for (int a = 0; a < D; ++a) q = fmaf(dl[t][a], v[a], q);            // D_ij^2 - D_i0^2
+        const float dij = sqrt_approx(fmaxf(d0sq + q, 0.f));
+        x[t] = -q * p.inv_tau * rcp_approx(fmaxf(dij + d0, 1e-30f));
+      }
+    }
+    float tt[KPL], lsum = 0.f;
+#pragma unroll
+    for (int t = 0; t < KPL; ++t) {
+      tt[t] = (FULL || cvalid[t]) ? expm1_small(x[t]) : 0.f;
+      lsum += tt[t];
+    }
+    const float tbar = group_sum<LPW>(lsum) * inv_k;
+    const float r = ok ? inv_k * rcp_approx(1.f + tbar) : 0.f;
+    const float ntr = -tbar * r;
+#pragma unroll
+    for (int t = 0; t < KPL; ++t) {
+      const float aij = (FULL || cvalid[t]) ? fmaf(tt[t], r, ntr) : 0.f;    // A_ij - 1/k = (t_ij - tbar_i) r_i
+      acc[t][0] += aij;
+#pragma unroll
+      for (int a = 0; a < D; ++a) acc[t][1 + a] = fmaf(aij, u[a], acc[t][1 + a]);
+    }
+#pragma unroll
+    for (int a = 0; a < D; ++a) uacc[a] += ok ? w[a] : 0.f;
+  };
+
+  // Scalar weights: a row farther than dmax2 from c_0 lies outside all centroids and is only counted; the others
+  // (about a fraction dmax2 / spread of the rows) take the general path, under a warp-uniform branch.
+  auto row_any = [&](const float (&w)[D], bool ok, auto full_tag) {
+    if constexpr (D == 1) {
+      const float u0 = w[0] - c0[0];
+      const bool fast = ok && (fabsf(u0) > dmax2);
+      const bool pos = fast && (u0 > 0.f), neg = fast && !(u0 > 0.f);
+      fx[0] += pos ? 1.f : 0.f;
+      fx[1] += pos ? w[0] : 0.f;
+      fx[2] += neg ? 1.f : 0.f;
+      fx[3] += neg ? w[0] : 0.f;
+      if (__any_sync(0xffffffffu, ok && !fast)) row(w, ok && !fast, full_tag);
+    } else {
+      row(w, ok, full_tag);
+    }
+  };
+
+  auto load_w = [&](long long grow, float (&w)[D]) {
+    if constexpr (D == 4) {
+      const float4 v4 = __ldg(reinterpret_cast<const float4*>(p.W) + grow);
+      w[0] = v4.x; w[1] = v4.y; w[2] = v4.z; w[3] = v4.w;
+    } else if constexpr (D == 2) {
+      const float2 v2 = __ldg(reinterpret_cast<const float2*>(p.W) + grow);
+      w[0] = v2.x; w[1] = v2.y;
+    } else {
+      w[0] = __ldg(p.W + grow);
+    }
+  };
+
+  for (int tile = t_lo; tile < t_hi; ++tile) {
+    while (p.lt.tile_off[layer + 1] <= tile) ++layer;
+    if (layer != cur_layer) {
+      if (cur_layer >= 0 && layer_active) flush(cur_layer);
+      cur_layer = layer;
+      layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[p.iter & 1] != 0) && (p.st[layer].fwd_iters == p.iter);
+      if (layer_active) {
+        const float* Cl = p.C + (size_t)layer * k * D;
+        inv_k = 1.f / (float)k;
+#pragma unroll
+        for (int a = 0; a < D; ++a) {
+          c0[a] = Cl[a];
+          uacc[a] = 0.f;
+          slots[(KPL * NA + a) * BLOCK + tid] = 0.f;
+        }
+        if constexpr (D == 1) {
+          float dm = 0.f;
+          for (int j = 1; j < k; ++j) dm = fmaxf(dm, fabsf(Cl[j] - c0[0]));
+          dmax2 = 2.f * dm;
+#pragma unroll
+          for (int q = 0; q < NEXTRA; ++q) {
+            fx[q] = 0.f;
+            slots[(KPL * NA + D + q) * BLOCK + tid] = 0.f;
+          }
+        }
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          const int j = gl * KPL + t;
+          cvalid[t] = (j < k);
+          double d2 = 0.0;
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const double dd = cvalid[t] ? (double)Cl[j * D + a] - (double)c0[a] : 0.0;
+            dl[t][a] = (float)dd;
+            d2 += dd * dd;
+          }
+          dl2[t] = (float)d2;
+#pragma unroll
+          for (int a = 0; a < NA; ++a) {
+            acc[t][a] = 0.f;
+            slots[(t * NA + a) * BLOCK + tid] = 0.f;
+          }
+        }
+        since_spill = 0;
+      }
+    }
+    if (!layer_active) continue;
+    const long long row0 = p.lt.row_off[layer];
+    const long long rows = p.lt.row_off[layer + 1] - row0;
+    const long long tb = (long long)(tile - p.lt.tile_off[layer]) * TILE;
+    const bool full = (k == Cfg::KP);
+    if constexpr (LPW == 1) {
+      // thread-per-weight: a thread takes VEC consecutive rows per 128-bit load, UN loads per trip, all issued first
+      constexpr int VEC = Cfg::VEC, UN = Cfg::UN;
+      const bool vec_ok = ((row0 * D) % 4 == 0);
+      float wv[UN][VEC][D];
+      int nv[UN];                       // rows of each load that exist (32-bit: the row loop compares against it)
+#pragma unroll
+      for (int un = 0; un < UN; ++un) {
+        const long long loc = tb + (long long)(un * BLOCK + tid) * VEC;
+        const long long left = rows - loc;
+        nv[un] = left >= VEC ? VEC : (left > 0 ? (int)left : 0);
+        const long long grow = row0 + loc;
+        if (vec_ok && loc + VEC <= rows) {
+          const float4 x4 = __ldg(reinterpret_cast<const float4*>(p.W + grow * D));
+          const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+          for (int v = 0; v < VEC; ++v)
+#pragma unroll
+            for (int a = 0; a < D; ++a) wv[un][v][a] = xs[v * D + a];
+        } else {
+#pragma unroll
+          for (int v = 0; v < VEC; ++v)
+#pragma unroll
+            for (int a = 0; a < D; ++a) wv[un][v][a] = (loc + v < rows) ? __ldg(p.W + (grow + v) * D + a) : 0.f;
+        }
+      }
+      if (full) {
+#pragma unroll
+        for (int un = 0; un < UN; ++un)
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) row_any(wv[un][v], v < nv[un], std::true_type{});
+      } else {
+#pragma unroll
+        for (int un = 0; un < UN; ++un)
+#pragma unroll
+          for (int v = 0; v < VEC; ++v) row_any(wv[un][v], v < nv[un], std::false_type{});
+      }
+    } else {
+      // group-per-weight: a group walks its own WPG consecutive rows, two fetched ahead
+      const long long gb = tb + (long long)grp * WPG;
+#pragma unroll 1
+      for (int q0 = 0; q0 < WPG; q0 += 2) {
+        float wv[2][D];
+        bool okq[2];
+#pragma unroll
+        for (int qq = 0; qq < 2; ++qq) {
+          const long long loc = gb + q0 + qq;
+          okq[qq] = (loc < rows);
+          load_w(row0 + (okq[qq] ? loc : 0), wv[qq]);
+        }
+        if (full) {
+#pragma unroll
+          for (int qq = 0; qq < 2; ++qq) row_any(wv[qq], okq[qq], std::true_type{});
+        } else {
+#pragma unroll
+          for (int qq = 0; qq < 2; ++qq) row_any(wv[qq], okq[qq], std::false_type{});
+        }
+      }
+    }
+    if (++since_spill >= Cfg::SPILL_TILES) {
+      spill();
+      since_spill = 0;
+    }
+  }
+  grid_release_dependents();
+  if (cur_layer >= 0 && layer_active) flush(cur_layer);
+}
+
+template <int D, int KPL, int LPW>
+__global__ void __launch_bounds__(BLOCK, DeltaCfg<D, KPL, LPW>::MIN_BLOCKS)
+idkm_step_delta(const __grid_constant__ PassParams p) {
+  grid_dependency_sync();
+  delta_body<D, KPL, LPW>(p);
+}
+
 // One launch per forward iteration instead of two, for the smallest thread-per-weight layouts, where the fp32 and
 // the fp64 step have the same register budget: every block first takes its tiles of the layers that step in fp32,
 // then its tiles of the layers that step in fp64 (own tile table, own partial-sum buffers: the two run side by side
@@ -1351,13 +1758,15 @@ struct DualParams {
   PassParams p;   // fp32 step
   PassParams q;   // fp64 step
 };
-template <int D, int KPL>
+// DELTA: the collapsing layers step in the fp32 increment form (delta_body) instead of fp64 (precise_body).
+template <int D, int KPL, bool DELTA>
 __global__ void __launch_bounds__(BLOCK, PreciseCfg<D, KPL, 1>::MIN_BLOCKS)
 idkm_step_dual(const __grid_constant__ DualParams dp) {
   grid_dependency_sync();
   pass_body<STEP, D, KPL, 1, false>(dp.p);
   __syncthreads();
-  precise_body<D, KPL, 1>(dp.q);
+  if constexpr (DELTA) delta_body<D, KPL, 1>(dp.q);
+  else precise_body<D, KPL, 1>(dp.q);
 }
 
 
@@ -1765,7 +2174,10 @@ struct SmallLoopEntry {
 };
 constexpr int N_SMALL_FAMILY = 4;
 // family index f: 0..7 -> supports k <= kpl*lpw
-constexpr int N_FAMILY = 9;
+constexpr int N_FAMILY = 11;
+constexpr int FAM_WIDE = 8;    // the alternative layout for the largest codebooks (see the tables in idkm_inst.cuh)
+constexpr int FAM_4x4 = 9;     // 4 centroids per lane on 4 lanes, 8 centroids per lane on 2 lanes: group layouts for
+constexpr int FAM_8x2 = 10;    // 16 centroids, picked by rule (pick_family), never by the first-fit search
 const KernelEntry* kernel_entry(int mode, int d, int family);
 int pick_family(int mode, int d, int k);
 

@@ -16,9 +16,9 @@ static cudaError_t launch_jacobian_tile(const PassParams& p, int grid, cudaStrea
 // (families 3-5: 16, 32, 64 centroids)
 extern const KernelEntry k_table_jacobian[3][N_FAMILY] = {
     {IDKM_JAC_ENTRY(1, 2), IDKM_JAC_ENTRY(1, 4), IDKM_JAC_ENTRY(1, 8), IDKM_JACT_ENTRY(1, 16), IDKM_JACT_ENTRY(1, 32),
-     IDKM_JACT_ENTRY(1, 64), IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY},
+     IDKM_JACT_ENTRY(1, 64), IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY},
     {IDKM_JAC_ENTRY(2, 2), IDKM_JAC_ENTRY(2, 4), IDKM_JACT_ENTRY(2, 8), IDKM_JACT_ENTRY(2, 16), IDKM_JACT_ENTRY(2, 32),
-     IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY},
+     IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY},
     {IDKM_JAC_ENTRY(4, 2), IDKM_JACT_ENTRY(4, 4), IDKM_JACT_ENTRY(4, 8), IDKM_JACT_ENTRY(4, 16), IDKM_NO_ENTRY,
-     IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY}};
+     IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY}};
 }

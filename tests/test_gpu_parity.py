@@ -327,3 +327,37 @@ def test_sweep_point_fixed_iterations(m, d, b, tau):
         outc = gpu_run(wc, mode="implicit", ctx=out["ctx"])
         assert_close(outc["dC"], refc["dC"], TOL_GRAD, "dC at common C", record=rec)
         assert_close(outc["dW"], refc["dW"], TOL_GRAD, "dW at common C", record=rec)
+
+
+# ----------------------------------------------------------------------------------------------------------------
+# collapsing layers: the fp32 increment-form step and the fp64 step
+# ----------------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("m,d,k", [(200001, 1, 2), (150000, 1, 4), (100003, 1, 16), (60000, 1, 256), (120000, 2, 4),
+                                   (90001, 2, 64), (100000, 4, 4), (80000, 4, 16), (50000, 4, 200)])
+def test_collapsing_layer_in_both_step_forms(m, d, k):
+    """tau above the weights' spread: after a few steps every centroid lies within a sliver of tau of the others and
+    the layer leaves the ordinary fp32 step.  Both forms of the step for such layers (fp32 increment form, the default,
+    and fp64) must give the oracle's centroids -- which differ from each other by far less than the weights' fp32
+    resolution -- to the stated tolerance, launch per iteration and (small codebooks) one launch for the whole loop."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(m, d, k, 0.1, std=0.02, seed=m + k, max_iter=5, adj_max_iter=3, init="rows")
+    ref = oracle_run(wl, want_dW=False)
+    spread = np.abs(ref["C"] - ref["C"].mean(0)).max()
+    assert spread < 1e-3 * wl.tau, spread              # the oracle's centroids have collapsed
+    W, C0 = torch.from_numpy(wl.W).cuda(), torch.from_numpy(wl.C0).cuda()
+    outs = {}
+    for form in (0, 1):
+        ctx = B.Context()
+        ctx.set_collapse_step(form)
+        ctx.set_forward_loop(1)
+        C = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter, want_Wq=False).C.cpu().numpy()
+        info = ctx.info()[0]
+        assert info.status == 0 and info.fwd_iters == wl.max_iter
+        assert_close(C, ref["C"], TOL_C, f"C, collapse step form {form}",
+                     record=f"collapsing layer m={m} d={d} k={k}, step form {form}")
+        # the differences BETWEEN centroids are what the ordinary fp32 step cannot resolve
+        assert_close(C - C.mean(0), ref["C"] - ref["C"].mean(0), 5e-4, f"centroid spread, form {form}")
+        assert abs(info.fwd_residual - ref["res"]) <= 2e-3 * ref["res"] + 1e-12
+        outs[form] = C
+    assert_close(outs[0], outs[1], TOL_C, "the two forms against each other")
