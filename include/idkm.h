@@ -318,8 +318,13 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
  * runs out the kernel returns and the layer's status is IDKM_ERR_TIMEOUT.  1: always one launch per iteration
  * (for the smallest codebooks -- k <= 4 at d = 1, k <= 2 at d = 2 -- that launch is a kernel that steps the fp32 and
  * the collapsing, fp64 layers of a batch side by side).  2: as 1, but the fp32 and the fp64 step of an iteration
- * are always two launches, one after the other.  All three run the same iteration; 0 differs from the others only by
- * the order of the cross-block sums, 1 and 2 give bitwise the same result.
+ * are always two launches, one after the other.  3: as 2, and for codebooks of at most 16 centroids the fp32 step
+ * receives its rows through a pipeline of bulk asynchronous copies into shared memory (one copy per trip, issued three
+ * trips ahead, completion on a shared-memory barrier with a bounded wait: if a copy never arrives the kernel returns
+ * and the layer's status is IDKM_ERR_TIMEOUT) instead of per-thread 128-bit loads; layers whose first row is not
+ * 16-byte aligned keep the loads.  All run the same iteration; 0 differs from the others only by the order of the
+ * cross-block sums, 1 and 2 give bitwise the same result, and so does 3 when as many blocks are resident with the
+ * copy stages in shared memory as without (otherwise the cross-block sums are grouped differently).
  */
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 

@@ -346,7 +346,8 @@ class Context:
 
     def set_forward_loop(self, method: int) -> None:
         """0: small layers run the whole forward loop in one cooperative launch (default); 1: a launch per iteration;
-        2: a launch per iteration and never the kernel that steps fp32 and fp64 layers side by side."""
+        2: a launch per iteration and never the kernel that steps fp32 and fp64 layers side by side; 3: as 2 with the
+        rows of small-codebook layers streamed by bulk asynchronous copies."""
         _check(lib.idkm_set_forward_loop(self._h, int(method)))
 
     def set_test_hooks(self, missing_arrivals: int = 0, spin_limit_ticks: int = 0) -> None:

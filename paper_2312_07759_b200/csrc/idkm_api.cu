@@ -31,6 +31,7 @@ extern const SmallLoopEntry k_table_small[3][N_SMALL_FAMILY];
 extern const DualEntry k_table_dual[3][2];
 extern const DualEntry k_table_dual_delta[3][2];
 extern const KernelEntry k_table_step_delta[3][N_FAMILY];
+extern const KernelEntry k_table_step_bulk[3][N_FAMILY];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
@@ -408,13 +409,27 @@ static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams
   const int mode64 = ctx->collapse_step == 0 ? STEP_DELTA : STEP_PRECISE;
   const int f32 = pick_family(STEP, ctx->d, ctx->k), f64 = pick_family(mode64, ctx->d, ctx->k);
   const KernelEntry* e32 = ctx_entry(ctx, STEP, f32);
+  // forward-loop method 3: the bulk-copy variant of the fp32 step where it exists (thread-per-weight layouts)
+  int bulk_per_sm = 0;
+  if (ctx->forward_loop == 3 && !ctx->squared && k_table_step_bulk[d_index(ctx->d)][f32].launch) {
+    e32 = &k_table_step_bulk[d_index(ctx->d)][f32];
+    (void)cudaFuncSetAttribute(e32->func, cudaFuncAttributeMaxDynamicSharedMemorySize, e32->dyn_smem);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bulk_per_sm, e32->func, BLOCK, e32->dyn_smem) != cudaSuccess || bulk_per_sm < 1) {
+      (void)cudaGetLastError();
+      bulk_per_sm = 1;
+    }
+  }
   const KernelEntry* e64 = kernel_entry(mode64, ctx->d, f64);
   static const bool dual_off = (getenv("IDKM_NO_DUAL") != nullptr);   // tuning knob: always two launches per iteration
-  const DualEntry* de = (dual_off || ctx->forward_loop == 2 || ctx->squared) ? nullptr
+  const DualEntry* de = (dual_off || ctx->forward_loop >= 2 || ctx->squared) ? nullptr
                                                                              : dual_entry(ctx->d, ctx->k, mode64 == STEP_DELTA);
   PassParams q = *p;
   int rc = build_table(ctx, STEP, f32, &p->lt);
   if (rc != IDKM_OK) return rc;
+  if (bulk_per_sm > 0 && ctx->n_layers == 1) {   // the stages take shared memory: fewer blocks may fit than the table assumed
+    const long long nbb = (long long)ctx->sms * (bulk_per_sm > MAX_BLOCKS_PER_SM ? MAX_BLOCKS_PER_SM : bulk_per_sm);
+    if (p->lt.n_blocks > nbb) p->lt.n_blocks = (int)nbb;
+  }
   rc = build_table(ctx, mode64, f64, &q.lt);
   if (rc != IDKM_OK) return rc;
   int dual_grid = 0;
@@ -971,7 +986,7 @@ int idkm_set_collapse_step(idkm_ctx* ctx, int method) {
 
 int idkm_set_forward_loop(idkm_ctx* ctx, int method) {
   if (!ctx) return IDKM_ERR_NULL;
-  if (method < 0 || method > 2) return IDKM_ERR_PARAM;
+  if (method < 0 || method > 3) return IDKM_ERR_PARAM;
   ctx->forward_loop = method;
   return IDKM_OK;
 }

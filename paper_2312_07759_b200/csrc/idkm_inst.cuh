@@ -62,6 +62,34 @@ static cudaError_t launch_precise(const PassParams& p, int grid, cudaStream_t st
     &launch_precise<D, KPL, LPW>, (const void*)&idkm_step_precise<D, KPL, LPW>, KPL, LPW,         \
         PreciseCfg<D, KPL, LPW>::TILE, PreciseCfg<D, KPL, LPW>::PLEN, 0                           \
   }
+// Bulk-copy variant of the forward step (thread-per-weight layouts only; see BULK in idkm_kernels.cuh): the stages
+// of the copy pipeline follow the second-level sums in dynamic shared memory.
+template <int D, int KPL>
+static cudaError_t launch_step_bulk(const PassParams& p, int grid, cudaStream_t stream) {
+  using Cfg = PassCfg<STEP, D, KPL, 1>;
+  constexpr int DYN = Cfg::DYN_SMEM + BULK_STAGES * Cfg::UNROLL * BLOCK * 16;
+  static bool configured = false;
+  if (!configured) {
+    const cudaError_t rc = cudaFuncSetAttribute(idkm_pass<STEP, D, KPL, 1, false, true>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, DYN);
+    if (rc != cudaSuccess) return rc;
+    configured = true;
+  }
+  return launch_pdl(idkm_pass<STEP, D, KPL, 1, false, true>, p, grid, DYN, stream);
+}
+#define IDKM_BULK_ENTRY(D, KPL)                                                                              \
+  {                                                                                                          \
+    &launch_step_bulk<D, KPL>, (const void*)&idkm_pass<STEP, D, KPL, 1, false, true>, KPL, 1,                \
+        PassCfg<STEP, D, KPL, 1>::TILE, PassCfg<STEP, D, KPL, 1>::PLEN,                                      \
+        PassCfg<STEP, D, KPL, 1>::DYN_SMEM + BULK_STAGES * PassCfg<STEP, D, KPL, 1>::UNROLL * BLOCK * 16     \
+  }
+#define IDKM_BULK_ROW(D)                                                                                     \
+  {                                                                                                          \
+    IDKM_BULK_ENTRY(D, 2), IDKM_BULK_ENTRY(D, 4), IDKM_BULK_ENTRY(D, 8), IDKM_BULK_ENTRY(D, 16),             \
+        IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY, IDKM_NO_ENTRY,            \
+        IDKM_NO_ENTRY                                                                                        \
+  }
+
 #define IDKM_PRECISE_ROW(D)                                                                       \
   {                                                                                               \
     IDKM_PRECISE_ENTRY(D, 2, 1), IDKM_PRECISE_ENTRY(D, 4, 1), IDKM_PRECISE_ENTRY(D, 8, 1),        \

@@ -545,6 +545,34 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   __syncthreads();
 }
 
+// ---- bulk asynchronous copies into shared memory, completion on an mbarrier --------------------------------------
+constexpr int BULK_STAGES = 3;
+constexpr int BULK_WAIT_POLLS = 1 << 22;   // polls of one wait before the block gives up (each poll may itself block
+                                           // for a hardware-defined slice): seconds, against microseconds of copy
+__device__ __forceinline__ unsigned smem_addr(const void* ptr) { return (unsigned)__cvta_generic_to_shared(ptr); }
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// dst: shared memory, 16-byte aligned; src: global memory, 16-byte aligned; bytes: a multiple of 16
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, unsigned bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_addr(dst)),
+               "l"(src), "r"(bytes), "r"(smem_addr(bar))
+               : "memory");
+}
+
 // ---- the pass ------------------------------------------------------------------------------------
 // RELEASE: let the next kernel of the stream be scheduled once this block's rows are done (the caller has already
 // waited for the previous kernel).  The dual step kernel runs this body with RELEASE = false and releases after its
@@ -552,7 +580,10 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
 // SQ: the squared-distance variant, D_ij = ||w_i - c_j||^2 in the softmax (the distance the clustering objectives of
 // Sections 3.1 / 3.2 are written in) and n_ij = dD_ij/dw_i = 2 (w_i - c_j): no square root, no reciprocal square
 // root, no kink at w_i = c_j.
-template <int MODE, int D, int KPL, int LPW, bool RELEASE, bool SQ = false>
+// BULK (forward step, thread-per-weight layouts): the rows of a trip arrive in shared memory by one bulk
+// asynchronous copy per trip (cp.async.bulk, completion on an mbarrier), issued by one thread BULK_STAGES trips ahead
+// of the arithmetic, instead of by per-thread 128-bit loads issued at the top of the trip.
+template <int MODE, int D, int KPL, int LPW, bool RELEASE, bool SQ = false, bool BULK = false>
 __device__ __forceinline__ void pass_body(const PassParams& p) {
   using Cfg = PassCfg<MODE, D, KPL, LPW>;
   constexpr int NACC = Cfg::NACC;
@@ -952,6 +983,57 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   };
   fetch(t_lo, layer);
 
+  // ---- bulk-copy pipeline (see BULK above): stages after the second-level sums in dynamic shared memory ----------
+  constexpr bool BULK_ON = BULK && (LPW == 1) && (MODE == STEP);
+  constexpr int STAGE_FLOATS = BULK_ON ? Cfg::UNROLL * BLOCK * 4 : 4;
+  __shared__ __align__(8) unsigned long long bfull[BULK_ON ? BULK_STAGES : 1];
+  float* bstage = slots + (ACCUM ? BLOCK * KPL * NA : 0);
+  int ptile = t_lo, player = layer;   // producer cursor (used by thread 0)
+  int cons_n = 0;                      // bulk trips consumed so far
+  (void)bfull; (void)bstage; (void)ptile; (void)player; (void)cons_n;
+  // The next trip at or after the producer cursor whose layer steps in this launch and whose rows start on a 16-byte
+  // boundary is copied into stage n % BULK_STAGES (trips of other layers are skipped; unaligned layers keep the
+  // per-thread loads).  The routing flags do not change while a launch runs, so producer and consumer agree.
+  auto bulk_issue = [&](int n) {
+    if constexpr (BULK_ON) {
+      while (ptile < t_hi) {
+        while (p.lt.tile_off[player + 1] <= ptile) ++player;
+        const int lim = (t_hi < p.lt.tile_off[player + 1]) ? t_hi : p.lt.tile_off[player + 1];
+        const int a = (lim - ptile < Cfg::UNROLL) ? lim - ptile : Cfg::UNROLL;
+        const int tl = ptile;
+        ptile += a;
+        const bool act = (p.st[player].fwd_done == 0) && (p.st[player].precise[p.iter & 1] == 0) &&
+                         (p.st[player].fwd_iters == p.iter);
+        const long long r0 = p.lt.row_off[player];
+        if (!act || (r0 * D) % 4 != 0) continue;
+        const long long rws = p.lt.row_off[player + 1] - r0;
+        const long long tb = (long long)(tl - p.lt.tile_off[player]) * TILE;
+        long long nrows = (long long)a * TILE;
+        if (nrows > rws - tb) nrows = rws - tb;
+        const unsigned bytes = (unsigned)(nrows * D * 4);
+        const unsigned ab = bytes & ~15u;
+        float* dst = bstage + (n % BULK_STAGES) * STAGE_FLOATS;
+        const float* src = p.W + (r0 + tb) * D;
+        for (unsigned q = ab / 4; q < bytes / 4; ++q) dst[q] = __ldg(src + q);   // at most three trailing floats
+        mbar_arrive_expect_tx(&bfull[n % BULK_STAGES], ab);
+        if (ab > 0) bulk_copy_g2s(dst, src, ab, &bfull[n % BULK_STAGES]);
+        return;
+      }
+    }
+  };
+  if constexpr (BULK_ON) {
+    if (tid == 0) {
+#pragma unroll
+      for (int q = 0; q < BULK_STAGES; ++q) mbar_init(&bfull[q], 1);
+      mbar_init_fence();
+    }
+    __syncthreads();
+    if (tid == 0) {
+#pragma unroll
+      for (int q = 0; q < BULK_STAGES; ++q) bulk_issue(q);
+    }
+  }
+
   // ---- persistent loop over this block's tiles -------------------------------------------------
   int adv = 1;   // tiles consumed per trip: 1, or up to UNROLL consecutive tiles of one layer (thread-per-weight)
   for (int tile = t_lo; tile < t_hi; tile += adv) {
@@ -1006,9 +1088,41 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
       float gv[UN][VEC][D];
       (void)gv;
       long long first[UN];
+      bool from_stage = false;
+      if constexpr (BULK_ON) {
+        if (vec_ok) {
+          // this trip's rows were copied to a stage: wait for the copy (bounded), take this thread's rows, hand the
+          // stage back and let thread 0 start the copy of the trip BULK_STAGES ahead
+          from_stage = true;
+          unsigned long long* bar = &bfull[cons_n % BULK_STAGES];
+          const unsigned parity = (unsigned)((cons_n / BULK_STAGES) & 1);
+          bool arrived = false;
+          for (int poll = 0; poll < BULK_WAIT_POLLS && !arrived; ++poll) arrived = mbar_try_wait(bar, parity);
+          const float* stg = bstage + (cons_n % BULK_STAGES) * STAGE_FLOATS;
+#pragma unroll
+          for (int un = 0; un < UN; ++un) {
+            const long long loc = (un < adv) ? tbase + (long long)(un * BLOCK + tid) * VEC : rows;
+            first[un] = loc;
+            const float4 x = *reinterpret_cast<const float4*>(stg + (un * BLOCK + tid) * 4);
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int v = 0; v < VEC; ++v)
+#pragma unroll
+              for (int a = 0; a < D; ++a) wv[un][v][a] = (arrived && loc + v < rows) ? xs[v * D + a] : 0.f;
+          }
+          if (__syncthreads_or(arrived ? 0 : 1)) {
+            // a copy never arrived: report it and leave (the layer's reduction is not completed, the layer stops)
+            if (tid == 0) p.st[layer].status = ST_TIMEOUT;
+            return;
+          }
+          if (tid == 0) bulk_issue(cons_n + BULK_STAGES);
+          ++cons_n;
+        }
+      }
       // issue all loads of the tile first
 #pragma unroll
       for (int un = 0; un < UN; ++un) {
+        if (from_stage) break;
         // trips shorter than UNROLL tiles mark the missing tiles as out of range
         const long long loc = (un < adv) ? tbase + (long long)(un * BLOCK + tid) * VEC : rows;
         first[un] = loc;
@@ -1166,11 +1280,11 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
 }
 
-template <int MODE, int D, int KPL, int LPW, bool SQ = false>
+template <int MODE, int D, int KPL, int LPW, bool SQ = false, bool BULK = false>
 __global__ void __launch_bounds__(BLOCK, PassCfg<MODE, D, KPL, LPW>::MIN_BLOCKS)
 idkm_pass(const __grid_constant__ PassParams p) {
   grid_dependency_sync();
-  pass_body<MODE, D, KPL, LPW, true, SQ>(p);
+  pass_body<MODE, D, KPL, LPW, true, SQ, BULK>(p);
 }
 
 

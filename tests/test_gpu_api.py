@@ -345,3 +345,57 @@ def test_dual_step_kernel_routes_collapsing_layers_like_two_launches():
     for l, lw in enumerate(WL.split_layers(wl)):
         r = oracle_run(lw, want_dW=False)
         assert_close(ref[l * k:(l + 1) * k], r["C"], TOL_C, f"layer {l} C")
+
+
+@pytest.mark.parametrize("d,k,m", [(1, 2, 50001), (1, 4, 1 << 20), (2, 2, 300001), (2, 4, 70000), (4, 2, 123457),
+                                   (4, 4, 65536), (1, 8, 99999), (4, 16, 40000), (1, 16, 5), (2, 8, 1023)])
+def test_bulk_copy_pipeline_gives_the_result_of_the_per_thread_loads(d, k, m):
+    """Forward-loop method 3 streams the rows of small-codebook layers into shared memory by bulk asynchronous copies
+    (one per trip, three trips ahead, completion on a barrier with a bounded wait); the arithmetic per row is that of
+    method 2 -- ragged tails, sizes below one tile and a tolerance-mode run included."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(m, d, min(k, m), 0.01, std=0.03, seed=m + k, max_iter=7, adj_max_iter=1, init="rows" if m >= k else "quantile")
+    W, C0 = torch.from_numpy(wl.W).cuda(), torch.from_numpy(wl.C0).cuda()
+    res = {}
+    for method in (2, 3):
+        ctx = B.Context()
+        ctx.set_forward_loop(method)
+        fr = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter)
+        torch.cuda.synchronize()
+        info = ctx.info()[0]
+        assert info.status == 0 and info.fwd_iters == wl.max_iter, info
+        assert ctx.busy_tickets() == 0
+        tol_C = ctx.forward(W, C0, wl.tau, 1e-4, 60, want_Wq=False).C.cpu().numpy()
+        res[method] = (fr.C.cpu().numpy(), fr.Wq.cpu().numpy(), tol_C, ctx.info()[0].fwd_iters)
+    # (the stages take shared memory, so fewer blocks may be resident and the cross-block sums may be grouped
+    # differently: equal to a few units in the last place, not always bitwise)
+    assert_close(res[3][0], res[2][0], 2e-6, "C")
+    assert_close(res[3][1], res[2][1], 2e-6, "Wq")
+    assert_close(res[3][2], res[2][2], 2e-6, "C, tolerance mode")
+    assert abs(res[2][3] - res[3][3]) <= 1
+
+
+def test_bulk_copy_pipeline_on_batched_layers_with_unaligned_offsets():
+    """Layers whose first row is not 16-byte aligned keep the per-thread loads inside the same launch; aligned ones
+    take the copies; collapsing layers leave for the other step kernel in mid-loop."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    rng = np.random.default_rng(4)
+    sizes = [4096, 1001, 37, 20000, 3, 8192, 50000]
+    offs = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    stds = [0.05, 0.05, 0.05, 0.008, 0.05, 0.05, 0.008]          # two layers collapse at tau = 0.02
+    W = np.concatenate([(rng.standard_normal((n, 1)) * s) for n, s in zip(sizes, stds)]).astype(np.float32)
+    k = 3
+    C0 = np.concatenate([WL.quantile_centroids(W[offs[l]:offs[l + 1]], k) for l in range(len(sizes))])
+    Wd, Cd = torch.from_numpy(W).cuda(), torch.from_numpy(C0).cuda()
+    out = {}
+    for method in (2, 3):
+        ctx = B.Context()
+        ctx.set_forward_loop(method)
+        C = ctx.forward(Wd, Cd, float(np.float32(0.02)), 0.0, 25, layer_offsets=[int(x) for x in offs], want_Wq=False).C
+        torch.cuda.synchronize()
+        assert all(i.status == 0 and i.fwd_iters == 25 for i in ctx.info())
+        assert ctx.busy_tickets() == 0
+        out[method] = C.cpu().numpy()
+    assert np.array_equal(out[2], out[3])          # batched calls launch the same grid in both methods
