@@ -162,6 +162,21 @@ def stored_traffic(workload_name):
     return {key: v["dram_bytes_read"] + v["dram_bytes_write"] for key, v in t.get("kernels", {}).items()}
 
 
+def store_traffic(workload_name, entries, source):
+    """Writes profiles/traffic_cfg4.json from figures read off an ncu capture: entries maps
+    "<pass>:<centroids per lane>x<lanes per weight>" to (dram__bytes_read.sum, dram__bytes_write.sum) of one launch.  The
+    sha256 of the kernel source goes with them, so that a later change of the kernels voids the figures."""
+    import hashlib
+    src = os.path.join(ROOT, "paper_2312_07759_b200", "csrc", "idkm_kernels.cuh")
+    with open(src, "rb") as f:
+        sha = hashlib.sha256(f.read()).hexdigest()
+    out = {"workload": workload_name, "kernel_source_sha256": sha, "source": source,
+           "kernels": {key: {"dram_bytes_read": float(r), "dram_bytes_write": float(w)} for key, (r, w) in entries.items()}}
+    with open(os.path.join(ROOT, "profiles", "traffic_cfg4.json"), "w") as f:
+        json.dump(out, f, indent=1)
+        f.write("\n")
+
+
 def time_oracle_sample(wl, rows: int, it_f: int, it_a: int):
     """Times the float64 oracle on the first `rows` rows of the workload: it_f forward iterations and it_a
     adjoint iterations (plus the final pass and the codebook gradient they need).  Returns
@@ -223,7 +238,19 @@ def main():
                     help="step of collapsing layers: 0 fp32 increment form (default), 1 fp64")
     ap.add_argument("--iters", type=int, default=0, help="override the forward and adjoint iteration counts "
                     "(short runs for profiler captures; the reported value is then not the configured workload's)")
+    ap.add_argument("--store-traffic", nargs="+", metavar="KEY=READ,WRITE", default=None,
+                    help="record dram bytes per launch read off an ncu capture of this workload's loop kernels, e.g. "
+                    "'idkm_pass<ADJ>:16x16=100764160,3399680' (no GPU work is done)")
     args = ap.parse_args()
+    if args.store_traffic:
+        entries = {}
+        for item in args.store_traffic:
+            key, val = item.split("=")
+            r, w = val.split(",")
+            entries[key] = (float(r), float(w))
+        store_traffic(make_workload(args.workload).name, entries,
+                      "ncu --set full captures summarised in profiles/adjoint_kernel_cfg4.txt and profiles/step_kernel_cfg4.txt")
+        return
     if args.warmup < 3:
         args.warmup = 3 if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -312,15 +339,15 @@ def main():
     path = B.describe_path(d, k, T_a, 0)
     traffic_table = stored_traffic(wl.name if args.iters == 0 else None)
 
-    def kernel_roofline(label, layout, kernel_ms, ops, share):
+    def kernel_roofline(label, layout, kernel_ms, ops, share, bytes_per_row):
         fp32_ops, sfu_ops = ops
-        t_hbm = (4.0 * d * m) / (peaks["hbm_gbs"] * 1e9)
+        t_hbm = (bytes_per_row * m) / (peaks["hbm_gbs"] * 1e9)
         fp32_peak = SM_COUNT * FP32_LANES_PER_SM * SM_MAX_MHZ * 1e6
         sfu_peak = SM_COUNT * SFU_LANES_PER_SM * SM_MAX_MHZ * 1e6
         t_fp32, t_sfu = pairs * fp32_ops / fp32_peak, pairs * sfu_ops / sfu_peak
         sec = kernel_ms * 1e-3
         if t_hbm >= max(t_fp32, t_sfu):
-            r = {"bound": "hbm", "achieved": 4.0 * d * m / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            r = {"bound": "hbm", "achieved": bytes_per_row * m / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                  "peak_source": f"MEASURED_PEAKS.json hbm_gbs ({which})"}
         elif t_fp32 >= t_sfu:
             r = {"bound": "alu", "achieved": pairs * fp32_ops / sec / 1e12, "peak": fp32_peak / 1e12,
@@ -334,6 +361,7 @@ def main():
         r["share_of_step"] = share
         r["roofline_ms"] = max(t_hbm, t_fp32, t_sfu) * 1e3
         r["fp32_ops_per_pair"], r["sfu_ops_per_pair"] = fp32_ops, sfu_ops
+        r["algorithmic_bytes_per_launch"] = bytes_per_row * m
         # dram__bytes_read.sum + dram__bytes_write.sum of one launch from the stored ncu capture of this kernel (ncu
         # flushes the caches before the launch, so this is the cold-L2 figure); null when none is stored for this
         # workload and layout, or when the kernel source has changed since the capture
@@ -343,11 +371,13 @@ def main():
 
     step_total = float(np.mean(step_ms))
     roof_step = kernel_roofline("idkm_pass<STEP> (fused forward step)", path["step_layout"], step_kernel_ms, pair_ops(d),
-                                ph["steps"] / step_total) if T_f > 0 and step_kernel_ms > 0 else None
+                                ph["steps"] / step_total, 4.0 * d) if T_f > 0 and step_kernel_ms > 0 else None
     roof_adj = None
     if T_a > 0 and adj_kernel_ms > 0 and path["adjoint_route"] == "fused passes":
+        # the group-per-weight adjoint layouts also read each row's cached softmax reference and normaliser (8 bytes)
         roof_adj = kernel_roofline("idkm_pass<ADJ> (fused adjoint step)", path["adjoint_layout"], adj_kernel_ms,
-                                   adjoint_pair_ops(d), ph["adjoint"] / step_total)
+                                   adjoint_pair_ops(d), ph["adjoint"] / step_total,
+                                   4.0 * d + (8.0 if path["adjoint_layout"][1] > 1 else 0.0))
     ranked = sorted([r for r in (roof_step, roof_adj) if r is not None], key=lambda r: -r["share_of_step"])
     roof = ranked[0] if ranked else None
     roof_second = ranked[1] if len(ranked) > 1 else None
