@@ -329,6 +329,15 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 
 /*
+ * Element type of the soft-quantised weights the forward writes: 0 (default) fp32, 1 bfloat16, 2 IEEE half.  With 1
+ * or 2 the Wq_out argument of idkm_forward* points to m * d two-byte elements (still 16-byte aligned, passed through the
+ * float* parameter) and receives the fp32 result of Wq = A C rounded to nearest even -- the form in which the
+ * quantised layer is fed to a half-precision network in the training loop of Algorithm 2.  Everything else (C, A, the
+ * backward) stays fp32; idkm_quantize_host* always exchange fp32.  Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_PARAM.
+ */
+int idkm_set_wq_dtype(idkm_ctx* ctx, int dtype);
+
+/*
  * How the forward step treats a COLLAPSING layer, i.e. one whose centroids all lie within 0.0625 tau of each other
  * (tau above the spread of the weights: every centroid slides into the mean).  There the update of C is decided by
  * attention differences far below fp32 resolution of w - c_j, so such layers leave the ordinary fp32 step.

@@ -74,6 +74,8 @@ lib.idkm_set_test_hooks.argtypes = [_vp, C.c_int, C.c_int64]
 lib.idkm_set_test_hooks.restype = C.c_int
 lib.idkm_count_busy_tickets.argtypes = [_vp, C.POINTER(C.c_int)]
 lib.idkm_count_busy_tickets.restype = C.c_int
+lib.idkm_set_wq_dtype.argtypes = [_vp, C.c_int]
+lib.idkm_set_wq_dtype.restype = C.c_int
 lib.idkm_set_collapse_step.argtypes = [_vp, C.c_int]
 lib.idkm_set_collapse_step.restype = C.c_int
 lib.idkm_set_distance.argtypes = [_vp, C.c_int]
@@ -196,6 +198,7 @@ class Context:
         self._ws = None
         self._keep = None
         self.n_layers = 0
+        self._wq_dtype = 0
 
     def close(self):
         if getattr(self, "_h", None):
@@ -235,7 +238,8 @@ class Context:
         if self._ws is None or self._ws.numel() < nbytes or self._ws.device != W.device:
             self._ws = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
         Cout = torch.empty_like(C0)
-        Wq = torch.empty_like(W) if want_Wq else None
+        wq_type = (torch.float32, torch.bfloat16, torch.float16)[self._wq_dtype]
+        Wq = torch.empty(W.shape, dtype=wq_type, device=W.device) if want_Wq else None
         A = torch.empty((m, k), dtype=torch.float32, device=W.device) if want_A else None
         offs = (C.c_int64 * (L + 1))(*[int(x) for x in layer_offsets])
         rc = lib.idkm_forward_batched(self._h, _ptr(W), offs, L, d, _ptr(C0), k, float(tau), float(tol), int(max_iter),
@@ -319,6 +323,12 @@ class Context:
         _check(rc)
         self.n_layers = L
         return Cout, Wq, dW, dC, list(infos)
+
+    def set_wq_dtype(self, dtype: int) -> None:
+        """``idkm_set_wq_dtype``: 0 = Wq in fp32 (default), 1 = bfloat16, 2 = float16; ``forward`` then returns Wq as a
+        tensor of that type."""
+        _check(lib.idkm_set_wq_dtype(self._h, int(dtype)))
+        self._wq_dtype = int(dtype)
 
     def set_collapse_step(self, method: int) -> None:
         """``idkm_set_collapse_step``: 0 = collapsing layers step in the fp32 increment form (default), 1 = in fp64."""

@@ -267,6 +267,7 @@ struct idkm_ctx {
   bool ev_ok;
   bool ev_fwd_set, ev_bwd_set;
   int squared;          // 1: squared-distance variant (idkm_set_distance)
+  int wq_dtype;         // element type of Wq_out: 0 fp32, 1 bf16, 2 fp16 (idkm_set_wq_dtype)
   int collapse_step;    // 0: collapsing layers step in the fp32 increment form; 1: in fp64 (idkm_set_collapse_step)
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
   int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never;
@@ -367,6 +368,7 @@ static void fill_params(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams* p)
   p->alpha = 1.f;
   p->k = ctx->k;
   p->squared = ctx->squared;
+  p->wq_dtype = ctx->wq_dtype;
 }
 
 // Loops with a tolerance are queued in chunks of RUN_CHUNK iterations.  After each chunk the host peeks at the pinned
@@ -870,8 +872,11 @@ int idkm_quantize_host_ex(idkm_ctx* ctx, const float* W_host, const int64_t* lay
   IDKM_TRY(cudaMemcpyAsync(dC0, C0_host, cn, cudaMemcpyHostToDevice, s));
   IDKM_TRY(cudaMemcpyAsync(dG, dWq_host, wn, cudaMemcpyHostToDevice, sc));
   IDKM_TRY(cudaEventRecord(ctx->hev[0], sc));
+  const int wq_dtype_saved = ctx->wq_dtype;
+  ctx->wq_dtype = 0;   // the host buffers of this entry point are fp32
   int rc = idkm_forward_batched(ctx, dW_, layer_offsets, n_layers, d, dC0, k, tau, tol, max_iter, dC, nullptr,
                                 Wq_out_host ? dWq : nullptr, ws, ws_bytes, s);
+  ctx->wq_dtype = wq_dtype_saved;
   if (rc != IDKM_OK) { cudaStreamSynchronize(s); cudaStreamSynchronize(sc); return rc; }
   // C and Wq go back on the copy stream while the backward runs
   IDKM_TRY(cudaEventRecord(ctx->hev[1], s));
@@ -974,6 +979,13 @@ int idkm_set_distance(idkm_ctx* ctx, int squared) {
   if (squared != 0 && squared != 1) return IDKM_ERR_PARAM;
   if (ctx->squared != squared) ctx->have_forward = false;   // a backward must follow a forward of the same variant
   ctx->squared = squared;
+  return IDKM_OK;
+}
+
+int idkm_set_wq_dtype(idkm_ctx* ctx, int dtype) {
+  if (!ctx) return IDKM_ERR_NULL;
+  if (dtype < 0 || dtype > 2) return IDKM_ERR_PARAM;
+  ctx->wq_dtype = dtype;
   return IDKM_OK;
 }
 

@@ -12,6 +12,8 @@
 // fp64 and applies the pass's epilogue (M-step and stop test; adjoint update; ...).  Results
 // are therefore bit-reproducible from run to run.
 #pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <type_traits>
@@ -80,7 +82,7 @@ struct LayerTable {
 struct PassParams {
   const float* W;
   const float* G;     // upstream gradient dL/dWq (GRAD, SCATTER)
-  float* Wq;          // FINAL (may be null)
+  void* Wq;           // FINAL (may be null); element type wq_dtype
   float* A;           // FINAL (may be null)
   float* dW;          // SCATTER
   float* C;           // [L][k][d] centroids, updated in place by STEP
@@ -105,6 +107,7 @@ struct PassParams {
   int max_iter;       // iteration cap of the loop (for the advisory status)
   int* host_flag;     // device view of a pinned host word, or null: set to call_id once every layer's loop has ended
   int call_id;
+  int wq_dtype;       // element type of Wq (FINAL): 0 fp32, 1 bf16, 2 fp16 (round to nearest even of the fp32 result)
   int squared;        // 1: squared-distance variant; its layers always step in the fp32 kernel (the fp64 step's
                       // short exponential series is derived for the Euclidean distance)
   int iter;           // index of this forward iteration: a layer is stepped only while fwd_iters == iter, so that
@@ -543,6 +546,37 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
     }
   }
   __syncthreads();
+}
+
+// Stores N consecutive elements of the soft-quantised weights, starting at element index `elem` of Wq, in the element
+// type the caller asked for (bf16 / fp16: the fp32 result rounded to nearest even).  `vec`: the N elements may go out
+// as one store (their byte offset is a multiple of the store width).
+template <int N>
+__device__ __forceinline__ void store_wq(void* base, long long elem, const float (&v)[N], int dtype, bool vec) {
+  if (dtype == 0) {
+    float* dst = static_cast<float*>(base) + elem;
+    if (vec && N == 4) *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[N > 1 ? 1 : 0], v[N > 2 ? 2 : 0], v[N > 3 ? 3 : 0]);
+    else if (vec && N == 2) *reinterpret_cast<float2*>(dst) = make_float2(v[0], v[N > 1 ? 1 : 0]);
+    else {
+#pragma unroll
+      for (int i = 0; i < N; ++i) dst[i] = v[i];
+    }
+    return;
+  }
+  unsigned short h[N];
+#pragma unroll
+  for (int i = 0; i < N; ++i)
+    h[i] = (dtype == 1) ? __bfloat16_as_ushort(__float2bfloat16_rn(v[i])) : __half_as_ushort(__float2half_rn(v[i]));
+  unsigned short* dst = static_cast<unsigned short*>(base) + elem;
+  if (vec && N == 4) {
+    *reinterpret_cast<uint2*>(dst) = make_uint2((unsigned)h[0] | ((unsigned)h[N > 1 ? 1 : 0] << 16),
+                                                (unsigned)h[N > 2 ? 2 : 0] | ((unsigned)h[N > 3 ? 3 : 0] << 16));
+  } else if (vec && N == 2) {
+    *reinterpret_cast<unsigned*>(dst) = (unsigned)h[0] | ((unsigned)h[N > 1 ? 1 : 0] << 16);
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; ++i) dst[i] = h[i];
+  }
 }
 
 // ---- bulk asynchronous copies into shared memory, completion on an mbarrier --------------------------------------
@@ -1168,7 +1202,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
           else process(wv[un][v], gdummy, loc + v < rows, grow + v, outv[v], make_float2(0.f, 0.f));
         }
         if constexpr (MODE == FINAL || MODE == SCATTER) {
-          float* dst = (MODE == FINAL) ? p.Wq : p.dW;
+          float* dst = (MODE == FINAL) ? static_cast<float*>(p.Wq) : p.dW;
           if (dst != nullptr) {
             if (vec_ok && loc + VEC <= rows) {
               float os[4];
@@ -1176,13 +1210,21 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
               for (int v = 0; v < VEC; ++v)
 #pragma unroll
                 for (int a = 0; a < D; ++a) os[v * D + a] = outv[v][a];
-              *reinterpret_cast<float4*>(dst + grow * D) = make_float4(os[0], os[1], os[2], os[3]);
+              if constexpr (MODE == FINAL) store_wq<4>(p.Wq, grow * D, os, p.wq_dtype, true);
+              else *reinterpret_cast<float4*>(dst + grow * D) = make_float4(os[0], os[1], os[2], os[3]);
             } else {
 #pragma unroll
               for (int v = 0; v < VEC; ++v)
                 if (loc + v < rows)
 #pragma unroll
-                  for (int a = 0; a < D; ++a) dst[(grow + v) * D + a] = outv[v][a];
+                  for (int a = 0; a < D; ++a) {
+                    if constexpr (MODE == FINAL) {
+                      const float one[1] = {outv[v][a]};
+                      store_wq<1>(p.Wq, (grow + v) * D + a, one, p.wq_dtype, false);
+                    } else {
+                      dst[(grow + v) * D + a] = outv[v][a];
+                    }
+                  }
             }
           }
         }
@@ -1229,9 +1271,10 @@ __device__ __forceinline__ void pass_body(const PassParams& p) {
         if constexpr (MODE == FINAL || MODE == SCATTER) grow = row0 + gbase + (ok ? t : 0);
         process(w, gi, ok, grow, outv, rstat);
         if constexpr (MODE == FINAL || MODE == SCATTER) {
-          float* dst = (MODE == FINAL) ? p.Wq : p.dW;
+          float* dst = (MODE == FINAL) ? static_cast<float*>(p.Wq) : p.dW;
           if (dst != nullptr && ok && gl == 0) {
-            if constexpr (D == 4) *reinterpret_cast<float4*>(dst + grow * 4) = make_float4(outv[0], outv[1], outv[2], outv[3]);
+            if constexpr (MODE == FINAL) store_wq<D>(p.Wq, grow * D, outv, p.wq_dtype, true);
+            else if constexpr (D == 4) *reinterpret_cast<float4*>(dst + grow * 4) = make_float4(outv[0], outv[1], outv[2], outv[3]);
             else if constexpr (D == 2) *reinterpret_cast<float2*>(dst + grow * 2) = make_float2(outv[0], outv[1]);
             else dst[grow] = outv[0];
           }

@@ -399,3 +399,29 @@ def test_bulk_copy_pipeline_on_batched_layers_with_unaligned_offsets():
         assert ctx.busy_tickets() == 0
         out[method] = C.cpu().numpy()
     assert np.array_equal(out[2], out[3])          # batched calls launch the same grid in both methods
+
+
+@pytest.mark.parametrize("m,d,k", [(5003, 1, 4), (4099, 2, 16), (30001, 4, 64), (7, 4, 3), (20000, 1, 256)])
+def test_half_precision_wq_is_the_rounded_fp32_result(m, d, k):
+    """idkm_set_wq_dtype: Wq written as bfloat16 / float16 equals the fp32 Wq of the same call rounded to nearest even,
+    bit for bit (ragged sizes and both store paths), and stays within half a unit in the last place of the oracle."""
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    wl = WL.single_layer(m, d, min(k, m), 0.012, std=0.03, seed=m + k, max_iter=6, adj_max_iter=2,
+                         init="rows" if m >= k else "quantile")
+    ref = oracle_run(wl)
+    W, C0, G = (torch.from_numpy(x).cuda() for x in (wl.W, wl.C0, wl.G))
+    ctx = B.Context()
+    full = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter).Wq
+    for dtype, ttype, eps in ((1, torch.bfloat16, 2.0 ** -8), (2, torch.float16, 2.0 ** -11)):
+        ctx.set_wq_dtype(dtype)
+        fr = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter)
+        assert fr.Wq.dtype == ttype and fr.Wq.shape == W.shape
+        assert torch.equal(fr.Wq, full.to(ttype))
+        err = np.abs(fr.Wq.float().cpu().numpy() - ref["Wq"])
+        assert np.all(err <= eps * np.abs(ref["Wq"]) + 1e-7)
+        dW, dC = ctx.backward(G, B.JFB, 0.0, 0, 1.0)          # the backward is unaffected
+        assert_close(dC.cpu().numpy(), oracle_run(wl, mode="jfb")["dC"], TOL_GRAD, "dC")
+    ctx.set_wq_dtype(0)
+    assert torch.equal(ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter).Wq, full)
+    assert B.lib.idkm_set_wq_dtype(ctx._h, 3) == B.ERR_PARAM
