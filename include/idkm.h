@@ -313,9 +313,18 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
  * launch: per
  * iteration every block publishes one fp64 partial, all blocks meet at a grid-wide barrier, and every block then
  * adds the partials in the same order and takes the M-step itself, so only the partials cross L2 inside the loop;
- * the loop leaves at the iteration whose stop test passes.  Everything else (batched layers, larger layers or
- * codebooks, max_iter < 2) takes one launch per iteration.  Every barrier wait is bounded (about a second): if one
- * runs out the kernel returns and the layer's status is IDKM_ERR_TIMEOUT.  1: always one launch per iteration
+ * the loop leaves at the iteration whose stop test passes.  Batched layers, and single layers beyond that size, with
+ * k <= 16 also run the whole loop in one cooperative launch (Algorithm 2 clusters every layer of the network before
+ * each minibatch: "for all layers"): per iteration every block steps its tiles of all layers -- the fp32 step for the
+ * layers that have not collapsed, the increment-form step for those that have -- exactly as the launch-per-iteration
+ * kernels do, then all blocks meet at a grid-wide barrier; the loop leaves at the first barrier at which every
+ * layer's loop has ended.  The default takes this launch where it was measured faster than a launch per iteration:
+ * batches, except small ones (under 2^22 rows) of the smallest codebooks and large ones of the widest layouts
+ * (d >= 2 with d k >= 16); method 4 takes it wherever the kernel exists, single large layers included.  Everything
+ * else (larger codebooks, max_iter < 2, the squared distance, the fp64 step for collapsing layers) takes one launch
+ * per iteration.  Every barrier wait is bounded (about a second): if one
+ * runs out the kernel returns and the status of the layer (of every layer of a batch) is IDKM_ERR_TIMEOUT.
+ * 1: always one launch per iteration
  * (for the smallest codebooks -- k <= 4 at d = 1, k <= 2 at d = 2 -- that launch is a kernel that steps the fp32 and
  * the collapsing, fp64 layers of a batch side by side).  2: as 1, but the fp32 and the fp64 step of an iteration
  * are always two launches, one after the other.  3: as 2, and for codebooks of at most 16 centroids the fp32 step
@@ -323,8 +332,10 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
  * trips ahead, completion on a shared-memory barrier with a bounded wait: if a copy never arrives the kernel returns
  * and the layer's status is IDKM_ERR_TIMEOUT) instead of per-thread 128-bit loads; layers whose first row is not
  * 16-byte aligned keep the loads.  All run the same iteration; 0 differs from the others only by the order of the
- * cross-block sums, 1 and 2 give bitwise the same result, and so does 3 when as many blocks are resident with the
- * copy stages in shared memory as without (otherwise the cross-block sums are grouped differently).
+ * cross-block sums (and, for the batched single launch, by spreading the tiles over the resident blocks only), 1 and
+ * 2 give bitwise the same result, and so does 3 when as many blocks are resident with the
+ * copy stages in shared memory as without (otherwise the cross-block sums are grouped differently).  4: as 0, and the
+ * single launch for every problem it exists for (k <= 16).  Returns IDKM_ERR_PARAM for other values.
  */
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 

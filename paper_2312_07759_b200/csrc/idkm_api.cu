@@ -32,6 +32,7 @@ extern const DualEntry k_table_dual[3][2];
 extern const DualEntry k_table_dual_delta[3][2];
 extern const KernelEntry k_table_step_delta[3][N_FAMILY];
 extern const KernelEntry k_table_step_bulk[3][N_FAMILY];
+extern const LoopEntry k_table_step_loop[3][4];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
@@ -159,6 +160,24 @@ static const DualEntry* dual_entry(int d, int k, bool delta = true) {
   return e->launch ? e : nullptr;
 }
 
+// The single-launch loop kernel of (d, k) for batched or large layers, or null: it exists for k <= 16 and is compiled
+// for the layouts the fp32 step and the increment-form step pick by default (a tuning override that forces another
+// layout switches it off).
+static const LoopEntry* loop_entry(int d, int k) {
+  const int di = d_index(d);
+  if (di < 0 || k < 1 || k > 16) return nullptr;
+  const int cls = k <= 2 ? 0 : (k <= 4 ? 1 : (k <= 8 ? 2 : 3));
+  const int f32 = pick_family(STEP, d, k), fq = pick_family(STEP_DELTA, d, k);
+  if (f32 < 0 || fq < 0) return nullptr;
+  const KernelEntry* a = kernel_entry(STEP, d, f32);
+  const KernelEntry* b = kernel_entry(STEP_DELTA, d, fq);
+  const int want_a[4][2] = {{2, 1}, {4, 1}, {8, 1}, {d == 1 ? 16 : 8, d == 1 ? 1 : 2}};
+  const int want_b[4][2] = {{2, 1}, {4, 1}, {8, 1}, {8, 2}};
+  if (a->kpl != want_a[cls][0] || a->lpw != want_a[cls][1] || b->kpl != want_b[cls][0] || b->lpw != want_b[cls][1]) return nullptr;
+  const LoopEntry* e = &k_table_step_loop[di][cls];
+  return e->launch ? e : nullptr;
+}
+
 struct WorkspaceLayout {
   size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, off_sync, total;
   size_t off_hist_fwd, off_hist_adj;
@@ -211,8 +230,9 @@ static bool make_layout(int64_t m_total, int d, int k, int n_layers, int sms, Wo
   w.off_sync = o;      o = align_up(o + 4 * sizeof(unsigned int), 256);   // barrier words of the single-launch loop
   w.off_hist_fwd = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
   w.off_hist_adj = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
-  const DualEntry* de = dual_entry(d, k);
-  // (the second half of the dual kernel is the fp64 step or the fp32 increment-form step: room for the larger partial)
+  // second set of partial buffers for the kernels that step the fp32 and the collapsing layers in one launch
+  const bool de = dual_entry(d, k) != nullptr || loop_entry(d, k) != nullptr;
+  // (the second half is the fp64 step or the fp32 increment-form step: room for the larger partial)
   const int plen64 = de ? kernel_entry(STEP_DELTA, d, pick_family(STEP_DELTA, d, k))->plen : 0;
   w.max_groups64 = de ? w.max_groups : 0;
   w.off_partials64 = o;  o = align_up(o + sizeof(double) * (size_t)w.max_slots * plen64, 256);
@@ -270,10 +290,11 @@ struct idkm_ctx {
   int wq_dtype;         // element type of Wq_out: 0 fp32, 1 bf16, 2 fp16 (idkm_set_wq_dtype)
   int collapse_step;    // 0: collapsing layers step in the fp32 increment form; 1: in fp64 (idkm_set_collapse_step)
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
-  int forward_loop;     // 0: a single small layer runs its whole forward loop in one cooperative launch; 1: never;
+  int forward_loop;     // 0: single-launch loops where they were measured faster; 4: wherever they exist; 1: never;
                         // 2: never, and the fp32 and fp64 steps of an iteration are always two launches
   int hook_missing_arrivals;      // host-side fault injection for the timeout path (idkm_set_test_hooks); 0 at rest
   long long hook_spin_limit;      // 0: the default bound
+  int loop_blocks[3][4];                 // the same for the batched single-launch loop kernels
   int small_blocks[3][N_SMALL_FAMILY];   // cached co-resident grid of the single-launch loop kernels (0 = not queried)
   // bounded run-ahead of the tolerance-mode loops: a pinned host word the device sets when all layers are done
   int* h_flag;
@@ -481,7 +502,7 @@ constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM c
 // Returns IDKM_OK after queueing the loop, 1 if this problem should take the launch-per-iteration path.
 static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p, int max_iter) {
   static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
-  if (env_off || ctx->forward_loop != 0 || ctx->n_layers != 1 || max_iter < 2 || ctx->squared) return 1;
+  if (env_off || (ctx->forward_loop != 0 && ctx->forward_loop != 4) || ctx->n_layers != 1 || max_iter < 2 || ctx->squared) return 1;
   const int di = d_index(ctx->d);
   int f = -1;
   for (int q = 0; q < N_SMALL_FAMILY; ++q)
@@ -526,6 +547,70 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   sp.missing_arrivals = ctx->hook_missing_arrivals;
   if (ctx->hook_spin_limit > 0 && ctx->hook_spin_limit < SMALL_SPIN_LIMIT) sp.spin_limit = ctx->hook_spin_limit;
   if (se->launch(sp, (int)grid, ctx->stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 1;   // nothing was queued: take the launch-per-iteration path
+  }
+  ++ctx->launches;
+  return IDKM_OK;
+}
+
+// The single-launch loop for what try_small_loop does not take: batched layers and single layers beyond its size, with
+// at most 16 centroids.  Returns IDKM_OK after queueing the loop, 1 if this problem should take the
+// launch-per-iteration path.
+static int try_batch_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p0, int max_iter) {
+  static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
+  if (env_off || (ctx->forward_loop != 0 && ctx->forward_loop != 4) || ctx->squared || ctx->collapse_step != 0 || max_iter < 2) return 1;
+  const LoopEntry* le = loop_entry(ctx->d, ctx->k);
+  if (!le) return 1;
+  // Where the single launch was measured against the launch per iteration (B200, 30 iterations; batches of 21 x 50 K,
+  // 8 x 1 M and a ResNet-18-like mix of rows): it takes batches, except (a) small batches of the smallest codebooks,
+  // where one launch per iteration already steps both kinds of layers (17.5 against 21 us per iteration at
+  // 21 x 50 K, d = 1, k = 2), and (b) large batches of the register-heavy layouts, where the joint kernel keeps
+  // fewer blocks resident than the fp32 step alone (d = 4, k = 8, 8 x 1 M: 205 against 169 us).  A single layer
+  // beyond try_small_loop's size keeps the launch per iteration (m = 2^24: 36 against 42 us at d = 1, k = 4).
+  // Forward-loop method 4 takes the single launch wherever its kernel exists.
+  if (ctx->forward_loop != 4) {
+    if (ctx->n_layers < 2) return 1;
+    const bool has_dual = dual_entry(ctx->d, ctx->k) != nullptr;
+    if (has_dual && ctx->m_total < (1LL << 22)) return 1;
+    if (ctx->d >= 2 && ctx->d * ctx->k >= 16 && ctx->m_total > (1LL << 22)) return 1;
+  }
+  const int di = d_index(ctx->d), cls = ctx->k <= 2 ? 0 : (ctx->k <= 4 ? 1 : (ctx->k <= 8 ? 2 : 3));
+  int& nb = ctx->loop_blocks[di][cls];
+  if (nb == 0) {
+    int coop = 0, per_sm = 0;
+    nb = -1;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
+        cudaFuncSetAttribute(le->func, cudaFuncAttributeMaxDynamicSharedMemorySize, le->dyn_smem > 0 ? le->dyn_smem : 1) == cudaSuccess &&
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, le->func, BLOCK, le->dyn_smem) == cudaSuccess && per_sm >= 1)
+      nb = ctx->sms * (per_sm > MAX_BLOCKS_PER_SM ? MAX_BLOCKS_PER_SM : per_sm);
+    (void)cudaGetLastError();
+  }
+  if (nb <= 0) return 1;
+  LoopParams lp;
+  memset(&lp, 0, sizeof(lp));
+  lp.p = p0;
+  lp.q = p0;
+  int rc = build_table(ctx, STEP, pick_family(STEP, ctx->d, ctx->k), &lp.p.lt);
+  if (rc != IDKM_OK) return rc;
+  rc = build_table(ctx, STEP_DELTA, pick_family(STEP_DELTA, ctx->d, ctx->k), &lp.q.lt);
+  if (rc != IDKM_OK) return rc;
+  // all blocks are resident at once: each table spreads its tiles over at most that many
+  const int cap = nb;
+  if (lp.p.lt.n_blocks > cap) lp.p.lt.n_blocks = cap;
+  if (lp.q.lt.n_blocks > cap) lp.q.lt.n_blocks = cap;
+  const int grid = lp.p.lt.n_blocks > lp.q.lt.n_blocks ? lp.p.lt.n_blocks : lp.q.lt.n_blocks;
+  char* ws = static_cast<char*>(ctx->workspace);
+  lp.q.partials = reinterpret_cast<double*>(ws + wl.off_partials64);
+  lp.q.gpartials = reinterpret_cast<double*>(ws + wl.off_gpartials64);
+  lp.q.gtickets = reinterpret_cast<unsigned int*>(ws + wl.off_gtickets64);
+  lp.p.host_flag = lp.q.host_flag = nullptr;
+  lp.sync = reinterpret_cast<unsigned int*>(ws + wl.off_sync);
+  lp.max_iter = max_iter;
+  lp.spin_limit = SMALL_SPIN_LIMIT;
+  lp.missing_arrivals = ctx->hook_missing_arrivals;
+  if (ctx->hook_spin_limit > 0 && ctx->hook_spin_limit < SMALL_SPIN_LIMIT) lp.spin_limit = ctx->hook_spin_limit;
+  if (le->launch(lp, grid, ctx->stream) != cudaSuccess) {
     (void)cudaGetLastError();
     return 1;   // nothing was queued: take the launch-per-iteration path
   }
@@ -676,6 +761,7 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
 
   nvtxRangePushA("idkm forward loop");
   int rc = try_small_loop(ctx, wl, p, max_iter);
+  if (rc == 1) rc = try_batch_loop(ctx, wl, p, max_iter);
   if (rc == 1) rc = launch_step_loop(ctx, wl, &p, max_iter);
   nvtxRangePop();
   if (rc != IDKM_OK) return rc;
@@ -998,7 +1084,7 @@ int idkm_set_collapse_step(idkm_ctx* ctx, int method) {
 
 int idkm_set_forward_loop(idkm_ctx* ctx, int method) {
   if (!ctx) return IDKM_ERR_NULL;
-  if (method < 0 || method > 3) return IDKM_ERR_PARAM;
+  if (method < 0 || method > 4) return IDKM_ERR_PARAM;
   ctx->forward_loop = method;
   return IDKM_OK;
 }

@@ -22,31 +22,6 @@ struct SmallCfg {
   static constexpr int DYN_SMEM = PLEN * BLOCK * 4;
 };
 
-// Bounded wait until the arrival counter has reached `target`.  Returns false if the wait ran out or another block
-// raised the error word.
-__device__ __forceinline__ bool small_barrier(unsigned int* sync, unsigned int target, long long spin_limit, int* s_ok) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    volatile unsigned int* vs = sync;
-    int ok = 1;
-    __threadfence();
-    atomicAdd(&sync[0], 1u);
-    const long long t0 = clock64();
-    while ((int)(vs[0] - target) < 0) {
-      if (vs[1] != 0u || clock64() - t0 > spin_limit) {
-        atomicExch(&sync[1], 1u);
-        ok = 0;
-        break;
-      }
-    }
-    if (vs[1] != 0u) ok = 0;
-    __threadfence();
-    *s_ok = ok;
-  }
-  __syncthreads();
-  return *s_ok != 0;
-}
-
 // CHUNKED: some thread has more than SMALL_CHUNK rows; its fp32 sums are then moved out every SMALL_CHUNK rows.
 template <int D, int KPL, bool CHUNKED>
 __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constant__ SmallLoopParams sp) {
