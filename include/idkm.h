@@ -318,9 +318,9 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
  * each minibatch: "for all layers"): per iteration every block steps its tiles of all layers -- the fp32 step for the
  * layers that have not collapsed, the increment-form step for those that have -- exactly as the launch-per-iteration
  * kernels do, then all blocks meet at a grid-wide barrier; the loop leaves at the first barrier at which every
- * layer's loop has ended.  The default takes this launch where it was measured faster than a launch per iteration:
- * batches, except small ones (under 2^22 rows) of the smallest codebooks and large ones of the widest layouts
- * (d >= 2 with d k >= 16); method 4 takes it wherever the kernel exists, single large layers included.  Everything
+ * layer's loop has ended.  The default takes this launch where it was measured faster than a launch per iteration
+ * (batches with 5..8 scalar centroids or 3..4 centroids at d = 2); method 4 takes it wherever the kernel exists,
+ * single large layers included.  Everything
  * else (larger codebooks, max_iter < 2, the squared distance, the fp64 step for collapsing layers) takes one launch
  * per iteration.  Every barrier wait is bounded (about a second): if one
  * runs out the kernel returns and the status of the layer (of every layer of a batch) is IDKM_ERR_TIMEOUT.

@@ -356,11 +356,10 @@ static int build_table(idkm_ctx* ctx, int mode, int family, LayerTable* lt) {
   long long nb = (long long)ctx->sms * blocks_per_sm(ctx, mode, ctx->d, family);
   if (mode == JACOBIAN && e->plen > JAC_SMALL_PLEN_MAX && nb > (long long)ctx->sms * JAC_TILE_BLOCKS_PER_SM)
     nb = (long long)ctx->sms * JAC_TILE_BLOCKS_PER_SM;   // the workspace holds this many matrix partials
-  // Batched loops: layers drop out of a loop at different times (converged, or handed to the other step kernel),
-  // and the blocks that own their tiles return at once.  With more blocks than fit on the GPU at a time the
-  // hardware scheduler backfills the freed slots with blocks of the layers that still run, instead of leaving SMs
-  // idle for the rest of the launch.
-  if (ctx->n_layers > 1 && (mode == STEP || mode == STEP_PRECISE || mode == STEP_DELTA || mode == ADJ)) nb = (long long)ctx->sms * MAX_BLOCKS_PER_SM;
+  // (Batched loops too get one resident wave of blocks.  More blocks than fit at a time -- so that the scheduler could
+  // backfill the slots of layers that have dropped out of the loop -- measured slower in every case tried: the
+  // ResNet-18-shaped batch 38.5 -> 31.9 us per iteration, a tolerance-mode batch of eight layers 1.52 -> 1.36 ms; what a
+  // block costs before and after its rows outweighs the idle slots.)
   if (nb > tiles) nb = tiles;
   lt->n_blocks = (int)nb;
   lt->pad = 0;
@@ -563,17 +562,16 @@ static int try_batch_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   const LoopEntry* le = loop_entry(ctx->d, ctx->k);
   if (!le) return 1;
   // Where the single launch was measured against the launch per iteration (B200, 30 iterations; batches of 21 x 50 K,
-  // 8 x 1 M and a ResNet-18-like mix of rows): it takes batches, except (a) small batches of the smallest codebooks,
-  // where one launch per iteration already steps both kinds of layers (17.5 against 21 us per iteration at
-  // 21 x 50 K, d = 1, k = 2), and (b) large batches of the register-heavy layouts, where the joint kernel keeps
-  // fewer blocks resident than the fp32 step alone (d = 4, k = 8, 8 x 1 M: 205 against 169 us).  A single layer
-  // beyond try_small_loop's size keeps the launch per iteration (m = 2^24: 36 against 42 us at d = 1, k = 4).
-  // Forward-loop method 4 takes the single launch wherever its kernel exists.
+  // 8 x 1 M and a ResNet-18-like mix of rows; both with one resident wave of blocks): it is faster only for 5..8
+  // scalar centroids (22 against 26, 33 against 40, 38 against 43 us per iteration) and for 3..4 centroids at d = 2
+  // (19.5 against 21.8 us on the small batch, level on the large ones); elsewhere the launch per iteration, whose
+  // next launch is scheduled while the epilogue of the last one drains, is level or ahead (d = 4, k = 8, 8 x 1 M: 84
+  // against 128 us -- the joint kernel keeps fewer blocks resident than the fp32 step alone).  Those two classes take
+  // the single launch by default; forward-loop method 4 takes it wherever its kernel exists.
   if (ctx->forward_loop != 4) {
     if (ctx->n_layers < 2) return 1;
-    const bool has_dual = dual_entry(ctx->d, ctx->k) != nullptr;
-    if (has_dual && ctx->m_total < (1LL << 22)) return 1;
-    if (ctx->d >= 2 && ctx->d * ctx->k >= 16 && ctx->m_total > (1LL << 22)) return 1;
+    const bool cls_a = (ctx->d == 1 && ctx->k > 4 && ctx->k <= 8), cls_b = (ctx->d == 2 && ctx->k > 2 && ctx->k <= 4);
+    if (!cls_a && !cls_b) return 1;
   }
   const int di = d_index(ctx->d), cls = ctx->k <= 2 ? 0 : (ctx->k <= 4 ? 1 : (ctx->k <= 8 ? 2 : 3));
   int& nb = ctx->loop_blocks[di][cls];

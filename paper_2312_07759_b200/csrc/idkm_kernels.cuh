@@ -640,6 +640,8 @@ __device__ __forceinline__ void pass_body(const PassParams& p, int iter_arg = IT
   // weight-vectors of a group per unrolled loop body: two in the forward passes (more independent work per warp);
   // one in the backward passes, whose register budget is already full (measured: 4 % faster than two)
   constexpr int WUNROLL = FWD ? 2 : 1;
+  // thread-per-weight forward step: runs of whole trips in a streamlined inner loop (see the tile loop)
+  constexpr bool STREAM_RUNS = (LPW == 1);
   // The adjoint step takes each row's softmax reference and normaliser from p.rowstat (written by the
   // codebook-gradient pass at the same centroids, with the same arithmetic, so the exponentials come out bit-equal):
   // no row minimum, no row sum, no cross-lane reduction before the exponentials and no reciprocal.
@@ -1124,6 +1126,52 @@ __device__ __forceinline__ void pass_body(const PassParams& p, int iter_arg = IT
     if constexpr (LPW == 1) {
       const bool vec_ok = ((row0 * D) % 4 == 0);
       constexpr int UN = Cfg::UNROLL;
+      // Forward step: a run of whole trips inside one layer (every row exists, rows start on a 16-byte boundary) is
+      // taken in one inner loop with a running pointer -- no tile, layer or range arithmetic per trip -- and the
+      // 128-bit loads of the next trip are issued before the arithmetic of the current one.
+      if constexpr (MODE == STEP && !BULK_ON && STREAM_RUNS) {
+        const int lim_r = (t_hi < p.lt.tile_off[layer + 1]) ? t_hi : p.lt.tile_off[layer + 1];
+        const long long by_rows = (rows - tbase) / ((long long)UN * TILE);
+        const int by_tiles = (lim_r - tile) / UN;
+        const int nfull = vec_ok ? (by_rows < (long long)by_tiles ? (int)by_rows : by_tiles) : 0;
+        if (nfull > 0) {
+          const float4* wp = reinterpret_cast<const float4*>(p.W + (row0 + tbase) * D) + tid;
+          float4 cur[UN], nxt[UN];
+#pragma unroll
+          for (int un = 0; un < UN; ++un) nxt[un] = cur[un] = __ldg(wp + un * BLOCK);
+#pragma unroll 1
+          for (int s = 0; s < nfull; ++s) {
+            wp += UN * BLOCK;
+            if (s + 1 < nfull) {
+#pragma unroll
+              for (int un = 0; un < UN; ++un) nxt[un] = __ldg(wp + un * BLOCK);
+            }
+#pragma unroll
+            for (int un = 0; un < UN; ++un) {
+              const float xs[4] = {cur[un].x, cur[un].y, cur[un].z, cur[un].w};
+#pragma unroll
+              for (int v = 0; v < VEC; ++v) {
+                float w1[D], g0[D], o0[D];
+#pragma unroll
+                for (int a = 0; a < D; ++a) {
+                  w1[a] = xs[v * D + a];
+                  g0[a] = 0.f;
+                }
+                process(w1, g0, true, 0, o0, make_float2(0.f, 0.f));
+              }
+            }
+            since_spill += UN;
+            if (since_spill >= Cfg::SPILL_TILES) {
+              spill();
+              since_spill = 0;
+            }
+#pragma unroll
+            for (int un = 0; un < UN; ++un) cur[un] = nxt[un];
+          }
+          adv = nfull * UN;
+          continue;
+        }
+      }
       float wv[UN][VEC][D];
       float gv[UN][VEC][D];
       (void)gv;
@@ -1850,6 +1898,51 @@ __device__ __forceinline__ void delta_body(const PassParams& p, int iter_arg = I
       // thread-per-weight: a thread takes VEC consecutive rows per 128-bit load, UN loads per trip, all issued first
       constexpr int VEC = Cfg::VEC, UN = Cfg::UN;
       const bool vec_ok = ((row0 * D) % 4 == 0);
+      // a run of whole tiles inside the layer: one inner loop with a running pointer, the next tile's loads issued
+      // before the current tile's arithmetic (as in the fp32 forward step)
+      {
+        const int lim_r = (t_hi < p.lt.tile_off[layer + 1]) ? t_hi : p.lt.tile_off[layer + 1];
+        const long long by_rows = (rows - tb) / TILE;
+        const int by_tiles = lim_r - tile;
+        const int nfull = vec_ok ? (by_rows < (long long)by_tiles ? (int)by_rows : by_tiles) : 0;
+        if (nfull > 0) {
+          auto run = [&](auto full_tag) {
+            const float4* wp = reinterpret_cast<const float4*>(p.W + (row0 + tb) * D) + tid;
+            float4 cur[UN], nxt[UN];
+#pragma unroll
+            for (int un = 0; un < UN; ++un) nxt[un] = cur[un] = __ldg(wp + un * BLOCK);
+#pragma unroll 1
+            for (int s2 = 0; s2 < nfull; ++s2) {
+              wp += UN * BLOCK;
+              if (s2 + 1 < nfull) {
+#pragma unroll
+                for (int un = 0; un < UN; ++un) nxt[un] = __ldg(wp + un * BLOCK);
+              }
+#pragma unroll
+              for (int un = 0; un < UN; ++un) {
+                const float xs[4] = {cur[un].x, cur[un].y, cur[un].z, cur[un].w};
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) {
+                  float w1[D];
+#pragma unroll
+                  for (int a = 0; a < D; ++a) w1[a] = xs[v * D + a];
+                  row_any(w1, true, full_tag);
+                }
+              }
+              if (++since_spill >= Cfg::SPILL_TILES) {
+                spill();
+                since_spill = 0;
+              }
+#pragma unroll
+              for (int un = 0; un < UN; ++un) cur[un] = nxt[un];
+            }
+          };
+          if (full) run(std::true_type{});
+          else run(std::false_type{});
+          tile += nfull - 1;
+          continue;
+        }
+      }
       float wv[UN][VEC][D];
       int nv[UN];                       // rows of each load that exist (32-bit: the row loop compares against it)
 #pragma unroll
