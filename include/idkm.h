@@ -356,7 +356,8 @@ int idkm_set_wq_dtype(idkm_ctx* ctx, int dtype);
  * differences -(D_ij - D_i0) / tau, the attention increments A_ij - 1/k and the sums of (A_ij - 1/k) and
  * (A_ij - 1/k) u_i are all small quantities evaluated to fp32 relative accuracy; the M-step is completed in fp64 from
  * those sums and sum_i u_i.  1: the same step with fp64 distances, exponentials and sums (about four times slower per
- * row; kept as the reference for the other).  Both realise Algorithm 1's steps 3-5 for such layers and agree with
+ * row; kept as the reference for the other; launches per iteration only, the one-launch loops are not taken).  Both
+ * realise Algorithm 1's steps 3-5 for such layers and agree with
  * the float64 oracle within the stated tolerance.  Returns IDKM_OK, IDKM_ERR_NULL or IDKM_ERR_PARAM.
  */
 int idkm_set_collapse_step(idkm_ctx* ctx, int method);

@@ -501,7 +501,10 @@ constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM c
 // Returns IDKM_OK after queueing the loop, 1 if this problem should take the launch-per-iteration path.
 static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p, int max_iter) {
   static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
-  if (env_off || (ctx->forward_loop != 0 && ctx->forward_loop != 4) || ctx->n_layers != 1 || max_iter < 2 || ctx->squared) return 1;
+  // (the loop kernel steps a collapsing layer in the fp32 increment form; the fp64 step exists as launches only)
+  if (env_off || (ctx->forward_loop != 0 && ctx->forward_loop != 4) || ctx->n_layers != 1 || max_iter < 2 || ctx->squared ||
+      ctx->collapse_step != 0)
+    return 1;
   const int di = d_index(ctx->d);
   int f = -1;
   for (int q = 0; q < N_SMALL_FAMILY; ++q)

@@ -16,7 +16,8 @@ constexpr int SMALL_CHUNK = 32;   // rows a thread adds into one fp32 accumulato
 template <int D, int KPL>
 struct SmallCfg {
   static constexpr int NA = D + 1;
-  static constexpr int PLEN = KPL * NA;
+  static constexpr int PLENK = KPL * NA;           // per-centroid sums
+  static constexpr int PLEN = PLENK + D;           // ... and the sum of the weights (increment-form iterations)
   static constexpr int CH = BLOCK / PLEN;          // chunks of partial rows added in parallel in the second level
   static constexpr int KD = KPL * D;
   static constexpr int DYN_SMEM = PLEN * BLOCK * 4;
@@ -26,9 +27,8 @@ struct SmallCfg {
 template <int D, int KPL, bool CHUNKED>
 __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constant__ SmallLoopParams sp) {
   using Cfg = SmallCfg<D, KPL>;
-  constexpr int NA = Cfg::NA, PLEN = Cfg::PLEN, CH = Cfg::CH, KD = Cfg::KD;
+  constexpr int NA = Cfg::NA, PLEN = Cfg::PLEN, PLENK = Cfg::PLENK, CH = Cfg::CH, KD = Cfg::KD;
   __shared__ float red[NWARP][PLEN];
-  __shared__ double redd[NWARP][PLEN];
   __shared__ double chunk[CH][PLEN];
   __shared__ double tot[PLEN];
   __shared__ float c_sm[KD > 0 ? KD : 1];   // the current centroids (every block holds the same values)
@@ -52,8 +52,8 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
   for (int t = 0; t < KPL; ++t)
 #pragma unroll
     for (int a = 0; a < D; ++a) c[t][a] = (t < k) ? c_sm[t * D + a] : PAD_COORD;
-  double ec[6];
-  exp_scaled_coeffs(sp.inv_tau_d, ec);
+  const float inv_tau = (float)sp.inv_tau_d;
+  const float inv_k = 1.f / (float)k;
   bool ok = true;
 
   for (int it = 0; it < sp.max_iter && !done; ++it) {
@@ -149,64 +149,138 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       __syncthreads();
       if (tid < PLEN) {
         double s = 0.0;
+        if (tid < PLENK) {
 #pragma unroll
-        for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
+          for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
+        }
         __stcg(mine + tid, s);
       }
     } else {
-      // fp64 rows for a collapsing layer: fp64 distances, a short Taylor exp around the distance to centroid 0 (all
-      // centroids lie within PRECISE_SPAN * tau of each other), fp64 sums
-      double accd[KPL][NA];
+      // A collapsing layer (all centroids within PRECISE_SPAN * tau of each other) steps in the fp32 increment form
+      // (see delta_body): with c_0 the reference, delta_j = c_j - c_0 and u_i = w_i - c_0, the logit differences
+      // x_ij = -(D_ij - D_i0) / tau and the attention increments A_ij - 1/k = (t_ij - tbar_i) / (k (1 + tbar_i)),
+      // t = exp(x) - 1, are formed to fp32 accuracy RELATIVE to delta; summed: dS_j, dN_j = sum (A_ij - 1/k) u_i and
+      // sum_i w_i.  The M-step below turns them into C+_j = c_0 + (U / k + dN_j) / (m / k + dS_j) in fp64.
+      float c0[D], dl[KPL][D], dl2[KPL];
 #pragma unroll
-      for (int t = 0; t < KPL; ++t)
+      for (int a = 0; a < D; ++a) c0[a] = c[0][a];
 #pragma unroll
-        for (int a = 0; a < NA; ++a) accd[t][a] = 0.0;
-      for (long long r = (long long)b * BLOCK + tid; r < m; r += (long long)G * BLOCK) {
-        float w[D];
-        load_row(r, w);
-        double wd[D], dist[KPL], e[KPL];
+      for (int t = 0; t < KPL; ++t) {
+        double d2 = 0.0;
 #pragma unroll
-        for (int a = 0; a < D; ++a) wd[a] = (double)w[a];
-#pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          double sq = 0.0;
-#pragma unroll
-          for (int a = 0; a < D; ++a) {
-            const double df = wd[a] - (double)c[t][a];
-            sq = (D == 1) ? fabs(df) : fma(df, df, sq);
-          }
-          dist[t] = (D == 1) ? sq : sqrt(sq);
+        for (int a = 0; a < D; ++a) {
+          const double dd = (t < k) ? (double)c[t][a] - (double)c0[a] : 0.0;
+          dl[t][a] = (float)dd;
+          d2 += dd * dd;
         }
-        double lsum = 0.0;
-#pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          e[t] = (t < k) ? exp_scaled(dist[0] - dist[t], ec) : 0.0;
-          lsum += e[t];
-        }
-        double rr = (double)rcp_approx((float)lsum);
-        rr = rr * (2.0 - lsum * rr);
-        rr = rr * (2.0 - lsum * rr);
-#pragma unroll
-        for (int t = 0; t < KPL; ++t) {
-          accd[t][0] = fma(e[t], rr, accd[t][0]);
-#pragma unroll
-          for (int a = 0; a < D; ++a) accd[t][1 + a] = fma(e[t], rr * wd[a], accd[t][1 + a]);
-        }
+        dl2[t] = (float)d2;
       }
+      float acc[KPL][NA], uacc[D];
 #pragma unroll
       for (int t = 0; t < KPL; ++t)
 #pragma unroll
         for (int a = 0; a < NA; ++a) {
-          double v = accd[t][a];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-          if (lane == 0) redd[warp][t * NA + a] = v;
+          acc[t][a] = 0.f;
+          if constexpr (CHUNKED) slots[(t * NA + a) * BLOCK + tid] = 0.f;
         }
+#pragma unroll
+      for (int a = 0; a < D; ++a) {
+        uacc[a] = 0.f;
+        if constexpr (CHUNKED) slots[(PLENK + a) * BLOCK + tid] = 0.f;
+      }
+      int since = 0;
+      const long long stride = (long long)G * BLOCK;
+      const long long r_first = (long long)b * BLOCK + tid;
+      float wn[D];
+#pragma unroll
+      for (int a = 0; a < D; ++a) wn[a] = 0.f;
+      if (r_first < m) load_row(r_first, wn);
+      for (long long r = r_first; r < m; r += stride) {
+        if constexpr (CHUNKED) {
+          if (since == SMALL_CHUNK) {
+#pragma unroll
+            for (int t = 0; t < KPL; ++t)
+#pragma unroll
+              for (int a = 0; a < NA; ++a) {
+                slots[(t * NA + a) * BLOCK + tid] += acc[t][a];
+                acc[t][a] = 0.f;
+              }
+#pragma unroll
+            for (int a = 0; a < D; ++a) {
+              slots[(PLENK + a) * BLOCK + tid] += uacc[a];
+              uacc[a] = 0.f;
+            }
+            since = 0;
+          }
+          ++since;
+        }
+        float w[D], u[D], x[KPL];
+#pragma unroll
+        for (int a = 0; a < D; ++a) {
+          w[a] = wn[a];
+          u[a] = w[a] - c0[a];
+        }
+        if (r + stride < m) load_row(r + stride, wn);
+        if constexpr (D == 1) {
+          // |u - delta| - |u| without forming u - delta: with s = sign(u), -s delta + 2 max(0, s delta - |u|)
+          const float aut = fabsf(u[0]) * inv_tau;
+          const float sg = copysignf(inv_tau, u[0]);
+#pragma unroll
+          for (int t = 0; t < KPL; ++t) {
+            const float sd = sg * dl[t][0];
+            x[t] = fmaf(-2.f, fmaxf(sd - aut, 0.f), sd);
+          }
+        } else {
+          float d0sq = 0.f, v[D];
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            d0sq = fmaf(u[a], u[a], d0sq);
+            v[a] = -2.f * u[a];
+          }
+          const float d0 = sqrt_approx(d0sq);
+#pragma unroll
+          for (int t = 0; t < KPL; ++t) {
+            float q = dl2[t];
+#pragma unroll
+            for (int a = 0; a < D; ++a) q = fmaf(dl[t][a], v[a], q);          // D_ij^2 - D_i0^2
+            const float dij = sqrt_approx(fmaxf(d0sq + q, 0.f));
+            x[t] = -q * inv_tau * rcp_approx(fmaxf(dij + d0, 1e-30f));
+          }
+        }
+        float tt[KPL], lsum = 0.f;
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          tt[t] = (t < k) ? expm1_small(x[t]) : 0.f;
+          lsum += tt[t];
+        }
+        const float tbar = lsum * inv_k;
+        const float rr = inv_k * rcp_approx(1.f + tbar);
+        const float ntr = -tbar * rr;
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) {
+          const float aij = (t < k) ? fmaf(tt[t], rr, ntr) : 0.f;
+          acc[t][0] += aij;
+#pragma unroll
+          for (int a = 0; a < D; ++a) acc[t][1 + a] = fmaf(aij, u[a], acc[t][1 + a]);
+        }
+#pragma unroll
+        for (int a = 0; a < D; ++a) uacc[a] += w[a];
+      }
+#pragma unroll
+      for (int o2 = 0; o2 < PLEN; ++o2) {
+        float v;
+        if (o2 < PLENK) v = acc[o2 / NA][o2 % NA];
+        else v = uacc[o2 - PLENK];
+        if constexpr (CHUNKED) v += slots[o2 * BLOCK + tid];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) red[warp][o2] = v;
+      }
       __syncthreads();
       if (tid < PLEN) {
         double s = 0.0;
 #pragma unroll
-        for (int wv = 0; wv < NWARP; ++wv) s += redd[wv][tid];
+        for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
         __stcg(mine + tid, s);
       }
     }
@@ -237,11 +311,16 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       (void)a;
       const bool own = (lane < k * D);
       double num = 0.0, den = 0.0, bad = 0.0, dead = 0.0, cq = 0.0;
+      // increment form: centroid 0 as it was when the rows were taken (read by all lanes before any lane writes)
+      const double c0a = (double)c_sm[own ? a : 0];
+      __syncwarp();
       if (own) {
-        const double s = tot[j * NA];
+        const double mk = (double)m / (double)k;
+        const double s = precise ? mk + tot[j * NA] : tot[j * NA];
         const bool alive = (s >= S_MIN);
         const double cold = (double)c_sm[lane];
-        const double cnew = alive ? tot[j * NA + 1 + a] / s : cold;
+        const double ubar = precise ? (tot[PLENK + a] - (double)m * c0a) / (double)k : 0.0;
+        const double cnew = alive ? (precise ? c0a + (ubar + tot[j * NA + 1 + a]) / s : tot[j * NA + 1 + a] / s) : cold;
         if (!alive && a == 0) dead = 1.0;
         if (!(s == s) || s > 1e300 || !(cnew == cnew) || fabs(cnew) > 1e300) bad = 1.0;
         num = (cnew - cold) * (cnew - cold);

@@ -347,17 +347,22 @@ def test_collapsing_layer_in_both_step_forms(m, d, k):
     assert spread < 1e-3 * wl.tau, spread              # the oracle's centroids have collapsed
     W, C0 = torch.from_numpy(wl.W).cuda(), torch.from_numpy(wl.C0).cuda()
     outs = {}
-    for form in (0, 1):
+    # (form, forward-loop method): increment form and fp64 by a launch per iteration, increment form in the one-launch loop
+    for form, method in ((0, 1), (1, 1), (0, 0)):
         ctx = B.Context()
         ctx.set_collapse_step(form)
-        ctx.set_forward_loop(1)
+        ctx.set_forward_loop(method)
+        n0 = ctx.launches
         C = ctx.forward(W, C0, wl.tau, 0.0, wl.max_iter, want_Wq=False).C.cpu().numpy()
+        if method == 0 and (k <= 8 or (k <= 16 and d <= 2)):
+            assert ctx.launches - n0 == 3            # init, the whole loop, final pass
         info = ctx.info()[0]
         assert info.status == 0 and info.fwd_iters == wl.max_iter
-        assert_close(C, ref["C"], TOL_C, f"C, collapse step form {form}",
-                     record=f"collapsing layer m={m} d={d} k={k}, step form {form}")
+        assert_close(C, ref["C"], TOL_C, f"C, collapse step form {form}, loop method {method}",
+                     record=f"collapsing layer m={m} d={d} k={k}, step form {form}" + (", one launch" if method == 0 else ""))
         # the differences BETWEEN centroids are what the ordinary fp32 step cannot resolve
-        assert_close(C - C.mean(0), ref["C"] - ref["C"].mean(0), 5e-4, f"centroid spread, form {form}")
+        assert_close(C - C.mean(0), ref["C"] - ref["C"].mean(0), 5e-4, f"centroid spread, form {form}, method {method}")
         assert abs(info.fwd_residual - ref["res"]) <= 2e-3 * ref["res"] + 1e-12
-        outs[form] = C
-    assert_close(outs[0], outs[1], TOL_C, "the two forms against each other")
+        outs[(form, method)] = C
+    assert_close(outs[(0, 1)], outs[(1, 1)], TOL_C, "the two forms against each other")
+    assert_close(outs[(0, 0)], outs[(0, 1)], TOL_C, "one launch against a launch per iteration")
