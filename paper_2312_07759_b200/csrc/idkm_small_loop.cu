@@ -70,43 +70,74 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
         w[0] = __ldg(sp.W + r);
       }
     };
-    if (!precise) {
-      // fp32 rows: the arithmetic of the fused forward step (Algorithm 1, steps 3-5)
-      float acc[KPL][NA];
+    // Sums of this thread: [t * NA + a] per centroid, then D entries for the sum of the weights (increment form only).
+    // A long fp32 running sum drops the many terms below half its ulp (one-sided): threads with more than
+    // SMALL_CHUNK rows move their sums into a private shared-memory slot every SMALL_CHUNK rows.
+    float sum[PLEN];
 #pragma unroll
-      for (int t = 0; t < KPL; ++t)
+    for (int o = 0; o < PLEN; ++o) {
+      sum[o] = 0.f;
+      if constexpr (CHUNKED) slots[o * BLOCK + tid] = 0.f;
+    }
+    int since = 0;
+    auto spill = [&]() {
 #pragma unroll
-        for (int a = 0; a < NA; ++a) {
-          acc[t][a] = 0.f;
-          if constexpr (CHUNKED) slots[(t * NA + a) * BLOCK + tid] = 0.f;
-        }
-      int since = 0;
+      for (int o = 0; o < PLEN; ++o) {
+        slots[o * BLOCK + tid] += sum[o];
+        sum[o] = 0.f;
+      }
+    };
+    // The rows of this block, grid-strided: 128-bit loads of 4 / D rows each, two in flight beyond the one being
+    // processed; what does not fill a 128-bit load (and everything, if W is not 16-byte aligned) by row.
+    auto walk = [&](auto&& row) {
+      constexpr int VEC = 4 / D;
       const long long stride = (long long)G * BLOCK;
-      const long long r_first = (long long)b * BLOCK + tid;
-      float wn[D];   // the next row, fetched while the current one is processed
+      long long first_by_row = 0;
+      if ((reinterpret_cast<size_t>(sp.W) & 15) == 0) {
+        const long long nvec = m / VEC;
+        const float4* W4 = reinterpret_cast<const float4*>(sp.W);
+        long long q = (long long)b * BLOCK + tid;
+        float4 cur = make_float4(0.f, 0.f, 0.f, 0.f), n1 = cur, n2 = cur;
+        if (q < nvec) cur = __ldg(W4 + q);
+        if (q + stride < nvec) n1 = __ldg(W4 + q + stride);
+        for (; q < nvec; q += stride) {
+          if (q + 2 * stride < nvec) n2 = __ldg(W4 + q + 2 * stride);
+          if constexpr (CHUNKED) {
+            if (since >= SMALL_CHUNK) {
+              spill();
+              since = 0;
+            }
+            since += VEC;
+          }
+          const float xs[4] = {cur.x, cur.y, cur.z, cur.w};
 #pragma unroll
-      for (int a = 0; a < D; ++a) wn[a] = 0.f;
-      if (r_first < m) load_row(r_first, wn);
-      for (long long r = r_first; r < m; r += stride) {
-        // A long fp32 running sum drops the many terms below half its ulp (one-sided): threads with more than
-        // SMALL_CHUNK rows move their sums into a private shared-memory slot every SMALL_CHUNK rows.
+          for (int v = 0; v < VEC; ++v) {
+            float w[D];
+#pragma unroll
+            for (int a = 0; a < D; ++a) w[a] = xs[v * D + a];
+            row(w);
+          }
+          cur = n1;
+          n1 = n2;
+        }
+        first_by_row = nvec * VEC;
+      }
+      for (long long r = first_by_row + (long long)b * BLOCK + tid; r < m; r += stride) {
+        float w[D];
+        load_row(r, w);
         if constexpr (CHUNKED) {
-          if (since == SMALL_CHUNK) {
-#pragma unroll
-            for (int t = 0; t < KPL; ++t)
-#pragma unroll
-              for (int a = 0; a < NA; ++a) {
-                slots[(t * NA + a) * BLOCK + tid] += acc[t][a];
-                acc[t][a] = 0.f;
-              }
+          if (since >= SMALL_CHUNK) {
+            spill();
             since = 0;
           }
           ++since;
         }
-        float w[D];
-#pragma unroll
-        for (int a = 0; a < D; ++a) w[a] = wn[a];
-        if (r + stride < m) load_row(r + stride, wn);
+        row(w);
+      }
+    };
+    if (!precise) {
+      // fp32 rows: the arithmetic of the fused forward step (Algorithm 1, steps 3-5)
+      walk([&](const float (&w)[D]) {
         float dist[KPL], e[KPL];
 #pragma unroll
         for (int t = 0; t < KPL; ++t) {
@@ -131,30 +162,11 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
         for (int a = 0; a < D; ++a) rw[a] = rr * w[a];
 #pragma unroll
         for (int t = 0; t < KPL; ++t) {
-          acc[t][0] = fmaf(e[t], rr, acc[t][0]);
+          sum[t * NA] = fmaf(e[t], rr, sum[t * NA]);
 #pragma unroll
-          for (int a = 0; a < D; ++a) acc[t][1 + a] = fmaf(e[t], rw[a], acc[t][1 + a]);
+          for (int a = 0; a < D; ++a) sum[t * NA + 1 + a] = fmaf(e[t], rw[a], sum[t * NA + 1 + a]);
         }
-      }
-#pragma unroll
-      for (int t = 0; t < KPL; ++t)
-#pragma unroll
-        for (int a = 0; a < NA; ++a) {
-          float v = acc[t][a];
-          if constexpr (CHUNKED) v += slots[(t * NA + a) * BLOCK + tid];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-          if (lane == 0) red[warp][t * NA + a] = v;
-        }
-      __syncthreads();
-      if (tid < PLEN) {
-        double s = 0.0;
-        if (tid < PLENK) {
-#pragma unroll
-          for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
-        }
-        __stcg(mine + tid, s);
-      }
+      });
     } else {
       // A collapsing layer (all centroids within PRECISE_SPAN * tau of each other) steps in the fp32 increment form
       // (see delta_body): with c_0 the reference, delta_j = c_j - c_0 and u_i = w_i - c_0, the logit differences
@@ -175,52 +187,10 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
         }
         dl2[t] = (float)d2;
       }
-      float acc[KPL][NA], uacc[D];
+      walk([&](const float (&w)[D]) {
+        float u[D], x[KPL];
 #pragma unroll
-      for (int t = 0; t < KPL; ++t)
-#pragma unroll
-        for (int a = 0; a < NA; ++a) {
-          acc[t][a] = 0.f;
-          if constexpr (CHUNKED) slots[(t * NA + a) * BLOCK + tid] = 0.f;
-        }
-#pragma unroll
-      for (int a = 0; a < D; ++a) {
-        uacc[a] = 0.f;
-        if constexpr (CHUNKED) slots[(PLENK + a) * BLOCK + tid] = 0.f;
-      }
-      int since = 0;
-      const long long stride = (long long)G * BLOCK;
-      const long long r_first = (long long)b * BLOCK + tid;
-      float wn[D];
-#pragma unroll
-      for (int a = 0; a < D; ++a) wn[a] = 0.f;
-      if (r_first < m) load_row(r_first, wn);
-      for (long long r = r_first; r < m; r += stride) {
-        if constexpr (CHUNKED) {
-          if (since == SMALL_CHUNK) {
-#pragma unroll
-            for (int t = 0; t < KPL; ++t)
-#pragma unroll
-              for (int a = 0; a < NA; ++a) {
-                slots[(t * NA + a) * BLOCK + tid] += acc[t][a];
-                acc[t][a] = 0.f;
-              }
-#pragma unroll
-            for (int a = 0; a < D; ++a) {
-              slots[(PLENK + a) * BLOCK + tid] += uacc[a];
-              uacc[a] = 0.f;
-            }
-            since = 0;
-          }
-          ++since;
-        }
-        float w[D], u[D], x[KPL];
-#pragma unroll
-        for (int a = 0; a < D; ++a) {
-          w[a] = wn[a];
-          u[a] = w[a] - c0[a];
-        }
-        if (r + stride < m) load_row(r + stride, wn);
+        for (int a = 0; a < D; ++a) u[a] = w[a] - c0[a];
         if constexpr (D == 1) {
           // |u - delta| - |u| without forming u - delta: with s = sign(u), -s delta + 2 max(0, s delta - |u|)
           const float aut = fabsf(u[0]) * inv_tau;
@@ -259,30 +229,28 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
 #pragma unroll
         for (int t = 0; t < KPL; ++t) {
           const float aij = (t < k) ? fmaf(tt[t], rr, ntr) : 0.f;
-          acc[t][0] += aij;
+          sum[t * NA] += aij;
 #pragma unroll
-          for (int a = 0; a < D; ++a) acc[t][1 + a] = fmaf(aij, u[a], acc[t][1 + a]);
+          for (int a = 0; a < D; ++a) sum[t * NA + 1 + a] = fmaf(aij, u[a], sum[t * NA + 1 + a]);
         }
 #pragma unroll
-        for (int a = 0; a < D; ++a) uacc[a] += w[a];
-      }
+        for (int a = 0; a < D; ++a) sum[PLENK + a] += w[a];
+      });
+    }
 #pragma unroll
-      for (int o2 = 0; o2 < PLEN; ++o2) {
-        float v;
-        if (o2 < PLENK) v = acc[o2 / NA][o2 % NA];
-        else v = uacc[o2 - PLENK];
-        if constexpr (CHUNKED) v += slots[o2 * BLOCK + tid];
+    for (int o2 = 0; o2 < PLEN; ++o2) {
+      float v = sum[o2];
+      if constexpr (CHUNKED) v += slots[o2 * BLOCK + tid];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) red[warp][o2] = v;
-      }
-      __syncthreads();
-      if (tid < PLEN) {
-        double s = 0.0;
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+      if (lane == 0) red[warp][o2] = v;
+    }
+    __syncthreads();
+    if (tid < PLEN) {
+      double s = 0.0;
 #pragma unroll
-        for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
-        __stcg(mine + tid, s);
-      }
+      for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
+      __stcg(mine + tid, s);
     }
     // ---- everyone has published: grid-wide barrier ----
     ok = small_barrier(sp.sync, (unsigned int)(it + 1) * (unsigned int)(G + sp.missing_arrivals), sp.spin_limit, &s_ok);
