@@ -308,34 +308,29 @@ size_t idkm_codes_bytes(int64_t m, int k);   /* ceil(m * idkm_code_bits(k) / 8);
 int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_per_s, void* cuda_stream);
 
 /*
- * How the forward loop (Algorithm 1) is launched.  0 (default): a single layer with k <= 16 (k <= 8 for d = 4) and
- * at most about 4.8 million rows (64 rows per thread of the co-resident grid) runs the WHOLE loop in one cooperative
- * launch: per
- * iteration every block publishes one fp64 partial, all blocks meet at a grid-wide barrier, and every block then
- * adds the partials in the same order and takes the M-step itself, so only the partials cross L2 inside the loop;
- * the loop leaves at the iteration whose stop test passes.  Batched layers, and single layers beyond that size, with
- * k <= 16 also run the whole loop in one cooperative launch (Algorithm 2 clusters every layer of the network before
- * each minibatch: "for all layers"): per iteration every block steps its tiles of all layers -- the fp32 step for the
- * layers that have not collapsed, the increment-form step for those that have -- exactly as the launch-per-iteration
- * kernels do, then all blocks meet at a grid-wide barrier; the loop leaves at the first barrier at which every
- * layer's loop has ended.  The default takes this launch where it was measured faster than a launch per iteration
- * (batches with 5..8 scalar centroids or 3..4 centroids at d = 2); method 4 takes it wherever the kernel exists,
- * single large layers included.  Everything
- * else (larger codebooks, max_iter < 2, the squared distance, the fp64 step for collapsing layers) takes one launch
- * per iteration.  Every barrier wait is bounded (about a second): if one
- * runs out the kernel returns and the status of the layer (of every layer of a batch) is IDKM_ERR_TIMEOUT.
- * 1: always one launch per iteration
+ * How the forward loop (Algorithm 1) is launched.  0 (default): layers with k <= 16 (k <= 8 for d = 4) run the WHOLE
+ * loop in one cooperative launch -- a single layer of at most about 4.8 million rows (64 rows per thread of the
+ * co-resident grid), or a batch of layers (Algorithm 2 clusters every layer of the network before each minibatch:
+ * "for all layers") of at most four times that in total (d = 4: the same as a single layer) and no more layers than
+ * the grid has blocks.  The blocks are dealt out to the layers in proportion to their rows, at least one each; per
+ * iteration every block publishes one fp64 partial of its layer, all blocks meet at a grid-wide barrier, and every
+ * block then adds its layer's partials in the same order and takes the M-step itself, so only the partials cross L2
+ * inside the loop.  A layer leaves the loop at the iteration whose stop test passes; a batch leaves at the first
+ * barrier at which every layer has.  Layers that collapse on the way step in the fp32 increment form (see
+ * idkm_set_collapse_step).  Everything else (larger layers, batches or codebooks, max_iter < 2, the squared
+ * distance, the fp64 step for collapsing layers) takes one launch per iteration.  Every barrier wait is bounded
+ * (about a second): if one runs out the kernel returns and the status of the layer (of every layer of a batch) is
+ * IDKM_ERR_TIMEOUT.  1: always one launch per iteration
  * (for the smallest codebooks -- k <= 4 at d = 1, k <= 2 at d = 2 -- that launch is a kernel that steps the fp32 and
- * the collapsing, fp64 layers of a batch side by side).  2: as 1, but the fp32 and the fp64 step of an iteration
+ * the collapsing layers of a batch side by side).  2: as 1, but the fp32 step and the step of the collapsing layers
  * are always two launches, one after the other.  3: as 2, and for codebooks of at most 16 centroids the fp32 step
  * receives its rows through a pipeline of bulk asynchronous copies into shared memory (one copy per trip, issued three
  * trips ahead, completion on a shared-memory barrier with a bounded wait: if a copy never arrives the kernel returns
  * and the layer's status is IDKM_ERR_TIMEOUT) instead of per-thread 128-bit loads; layers whose first row is not
  * 16-byte aligned keep the loads.  All run the same iteration; 0 differs from the others only by the order of the
- * cross-block sums (and, for the batched single launch, by spreading the tiles over the resident blocks only), 1 and
- * 2 give bitwise the same result, and so does 3 when as many blocks are resident with the
- * copy stages in shared memory as without (otherwise the cross-block sums are grouped differently).  4: as 0, and the
- * single launch for every problem it exists for (k <= 16).  Returns IDKM_ERR_PARAM for other values.
+ * cross-block sums, 1 and 2 give bitwise the same result, and so does 3 when as many blocks are resident with the
+ * copy stages in shared memory as without (otherwise the cross-block sums are grouped differently).  Returns
+ * IDKM_ERR_PARAM for other values.
  */
 int idkm_set_forward_loop(idkm_ctx* ctx, int method);
 

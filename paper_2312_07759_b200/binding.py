@@ -355,10 +355,9 @@ class Context:
         return np.frombuffer(buf, dtype=np.float32, count=n.value).copy()
 
     def set_forward_loop(self, method: int) -> None:
-        """0: small layers run the whole forward loop in one cooperative launch (default); 1: a launch per iteration;
+        """0: small layers and batches of them run the whole forward loop in one cooperative launch (default); 1: a launch per iteration;
         2: a launch per iteration and never the kernel that steps fp32 and fp64 layers side by side; 3: as 2 with the
-        rows of small-codebook layers streamed by bulk asynchronous copies; 4: as 0, and the single launch for every
-        batch or layer with k <= 16, also where the default prefers a launch per iteration."""
+        rows of small-codebook layers streamed by bulk asynchronous copies."""
         _check(lib.idkm_set_forward_loop(self._h, int(method)))
 
     def set_test_hooks(self, missing_arrivals: int = 0, spin_limit_ticks: int = 0) -> None:

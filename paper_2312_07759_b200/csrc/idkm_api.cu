@@ -32,7 +32,6 @@ extern const DualEntry k_table_dual[3][2];
 extern const DualEntry k_table_dual_delta[3][2];
 extern const KernelEntry k_table_step_delta[3][N_FAMILY];
 extern const KernelEntry k_table_step_bulk[3][N_FAMILY];
-extern const LoopEntry k_table_step_loop[3][4];
 
 // Initialise the per-layer state and copy C0 into the working centroids.
 __global__ void idkm_init_forward(LayerState* st, int n_layers, const float* C0, float* C, int n_coord, int k, int d,
@@ -160,24 +159,6 @@ static const DualEntry* dual_entry(int d, int k, bool delta = true) {
   return e->launch ? e : nullptr;
 }
 
-// The single-launch loop kernel of (d, k) for batched or large layers, or null: it exists for k <= 16 and is compiled
-// for the layouts the fp32 step and the increment-form step pick by default (a tuning override that forces another
-// layout switches it off).
-static const LoopEntry* loop_entry(int d, int k) {
-  const int di = d_index(d);
-  if (di < 0 || k < 1 || k > 16) return nullptr;
-  const int cls = k <= 2 ? 0 : (k <= 4 ? 1 : (k <= 8 ? 2 : 3));
-  const int f32 = pick_family(STEP, d, k), fq = pick_family(STEP_DELTA, d, k);
-  if (f32 < 0 || fq < 0) return nullptr;
-  const KernelEntry* a = kernel_entry(STEP, d, f32);
-  const KernelEntry* b = kernel_entry(STEP_DELTA, d, fq);
-  const int want_a[4][2] = {{2, 1}, {4, 1}, {8, 1}, {d == 1 ? 16 : 8, d == 1 ? 1 : 2}};
-  const int want_b[4][2] = {{2, 1}, {4, 1}, {8, 1}, {8, 2}};
-  if (a->kpl != want_a[cls][0] || a->lpw != want_a[cls][1] || b->kpl != want_b[cls][0] || b->lpw != want_b[cls][1]) return nullptr;
-  const LoopEntry* e = &k_table_step_loop[di][cls];
-  return e->launch ? e : nullptr;
-}
-
 struct WorkspaceLayout {
   size_t off_state, off_S, off_F, off_g, off_u, off_partials, off_gpartials, off_gtickets, off_sync, total;
   size_t off_hist_fwd, off_hist_adj;
@@ -230,8 +211,8 @@ static bool make_layout(int64_t m_total, int d, int k, int n_layers, int sms, Wo
   w.off_sync = o;      o = align_up(o + 4 * sizeof(unsigned int), 256);   // barrier words of the single-launch loop
   w.off_hist_fwd = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
   w.off_hist_adj = o;  o = align_up(o + sizeof(float) * (size_t)n_layers * HIST_CAP, 256);
-  // second set of partial buffers for the kernels that step the fp32 and the collapsing layers in one launch
-  const bool de = dual_entry(d, k) != nullptr || loop_entry(d, k) != nullptr;
+  // second set of partial buffers for the kernel that steps the fp32 and the collapsing layers in one launch
+  const bool de = dual_entry(d, k) != nullptr;
   // (the second half is the fp64 step or the fp32 increment-form step: room for the larger partial)
   const int plen64 = de ? kernel_entry(STEP_DELTA, d, pick_family(STEP_DELTA, d, k))->plen : 0;
   w.max_groups64 = de ? w.max_groups : 0;
@@ -290,11 +271,10 @@ struct idkm_ctx {
   int wq_dtype;         // element type of Wq_out: 0 fp32, 1 bf16, 2 fp16 (idkm_set_wq_dtype)
   int collapse_step;    // 0: collapsing layers step in the fp32 increment form; 1: in fp64 (idkm_set_collapse_step)
   int adjoint_method;   // 0: explicit Jacobian where k d <= 8, fused passes otherwise; 1: always fused passes
-  int forward_loop;     // 0: single-launch loops where they were measured faster; 4: wherever they exist; 1: never;
+  int forward_loop;     // 0: small layers and batches of them run the whole forward loop in one cooperative launch; 1: never;
                         // 2: never, and the fp32 and fp64 steps of an iteration are always two launches
   int hook_missing_arrivals;      // host-side fault injection for the timeout path (idkm_set_test_hooks); 0 at rest
   long long hook_spin_limit;      // 0: the default bound
-  int loop_blocks[3][4];                 // the same for the batched single-launch loop kernels
   int small_blocks[3][N_SMALL_FAMILY];   // cached co-resident grid of the single-launch loop kernels (0 = not queried)
   // bounded run-ahead of the tolerance-mode loops: a pinned host word the device sets when all layers are done
   int* h_flag;
@@ -489,11 +469,15 @@ static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams
   return IDKM_OK;
 }
 
-// The single-launch loop takes a single layer with k <= 16 (k <= 8 for d = 4) whose rows fit SMALL_ROWS_PER_THREAD per
-// thread of the co-resident grid -- about 4.8 million rows on a 148-SM part (beyond that the tiled step kernels with
-// their deeper load pipelines are faster).  Blocks get at least SMALL_MIN_ROWS_PER_THREAD rows per thread: tiny layers use few blocks, which keeps
-// the cross-block sum short.
+// The single-launch loop of idkm_small_loop.cu takes layers with k <= 16 (k <= 8 for d = 4): a single layer whose rows
+// fit SMALL_ROWS_PER_THREAD per thread of the co-resident grid -- about 4.8 million rows on a 148-SM part (beyond that
+// the tiled step kernels with their deeper load pipelines are as fast) -- or a batch of up to as many layers as the grid
+// has blocks, with up to SMALL_BATCH_ROWS_PER_THREAD rows per thread (a batch pays more per iteration on the tiled path:
+// every block there walks several layers, each with its own chain of block sums and tickets).  The blocks are dealt out
+// to the layers in proportion to their rows, at least one each, and at least SMALL_MIN_ROWS_PER_THREAD rows per thread:
+// tiny layers use few blocks, which keeps the cross-block sum short.
 constexpr int SMALL_ROWS_PER_THREAD = 64;
+constexpr int SMALL_BATCH_ROWS_PER_THREAD = 256;
 constexpr int SMALL_CHUNK_ROWS = 32;   // threads with more rows than this move their fp32 sums out every 32 rows
 constexpr int SMALL_MIN_ROWS_PER_THREAD = 4;
 constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM clock ticks per barrier wait
@@ -502,8 +486,7 @@ constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM c
 static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p, int max_iter) {
   static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
   // (the loop kernel steps a collapsing layer in the fp32 increment form; the fp64 step exists as launches only)
-  if (env_off || (ctx->forward_loop != 0 && ctx->forward_loop != 4) || ctx->n_layers != 1 || max_iter < 2 || ctx->squared ||
-      ctx->collapse_step != 0)
+  if (env_off || ctx->forward_loop != 0 || max_iter < 2 || ctx->squared || ctx->collapse_step != 0)
     return 1;
   const int di = d_index(ctx->d);
   int f = -1;
@@ -522,16 +505,53 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
     (void)cudaGetLastError();
   }
   if (nb <= 0) return 1;
+  const int L = ctx->n_layers;
   const long long m = ctx->m_total;
-  if (m > (long long)SMALL_ROWS_PER_THREAD * nb * BLOCK) return 1;
+  if (L > nb || L > MAX_LAYERS) return 1;
+  // (d = 4 batches beyond the single-layer size measured slower than a launch per iteration: 8 x 1 M rows, 65 against 41 us)
+  if (m > (long long)((L == 1 || ctx->d == 4) ? SMALL_ROWS_PER_THREAD : SMALL_BATCH_ROWS_PER_THREAD) * nb * BLOCK) return 1;
   long long grid = (m + (long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK - 1) / ((long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK);
   if (grid > nb) grid = nb;
-  if (grid < 1) grid = 1;
+  if (grid < L) grid = L;
   if (2 * grid > wl.max_slots) return 1;   // the two partial buffers live in the partial-slot region
   SmallLoopParams sp;
   memset(&sp, 0, sizeof(sp));
   sp.W = ctx->W;
-  sp.m = m;
+  sp.n_layers = L;
+  // blocks per layer: one each, the rest in proportion to the rows (largest remainders first)
+  int cnt[MAX_LAYERS];
+  long long rem[MAX_LAYERS];
+  int given = 0;
+  const long long spare = grid - L;
+  for (int l = 0; l < L; ++l) {
+    const long long rows = ctx->row_off[l + 1] - ctx->row_off[l];
+    const long long share = (m > 0) ? spare * rows / m : 0;
+    cnt[l] = 1 + (int)share;
+    rem[l] = (m > 0) ? spare * rows % m : 0;
+    given += cnt[l];
+    sp.row_off[l] = ctx->row_off[l];
+  }
+  sp.row_off[L] = ctx->row_off[L];
+  while (given < grid) {
+    int best = 0;
+    for (int l = 1; l < L; ++l)
+      if (rem[l] > rem[best]) best = l;
+    ++cnt[best];
+    rem[best] = -1;
+    ++given;
+  }
+  long long max_rows_per_thread = 0;
+  sp.blk_first[0] = 0;
+  for (int l = 0; l < L; ++l) {
+    sp.blk_first[l + 1] = sp.blk_first[l] + cnt[l];
+    const long long rows = ctx->row_off[l + 1] - ctx->row_off[l];
+    const long long per = (rows + (long long)cnt[l] * BLOCK - 1) / ((long long)cnt[l] * BLOCK);
+    if (per > max_rows_per_thread) max_rows_per_thread = per;
+  }
+  for (int l = L + 1; l <= MAX_LAYERS; ++l) {
+    sp.blk_first[l] = sp.blk_first[L];
+    sp.row_off[l] = sp.row_off[L];
+  }
   sp.C = ctx->C;
   sp.st = p.st;
   sp.partials = p.partials;
@@ -542,76 +562,13 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   sp.inv_tau_d = p.inv_tau_d;
   sp.max_iter = max_iter;
   sp.hist = p.hist_fwd;
-  sp.chunked = (m > (long long)SMALL_CHUNK_ROWS * grid * BLOCK) ? 1 : 0;
+  sp.chunked = (max_rows_per_thread > SMALL_CHUNK_ROWS) ? 1 : 0;
   sp.spin_limit = SMALL_SPIN_LIMIT;
   // Host-side fault injection for tests of the timeout path (idkm_set_test_hooks; no GPU fault involved: the waits
   // are bounded and the kernel returns)
   sp.missing_arrivals = ctx->hook_missing_arrivals;
   if (ctx->hook_spin_limit > 0 && ctx->hook_spin_limit < SMALL_SPIN_LIMIT) sp.spin_limit = ctx->hook_spin_limit;
   if (se->launch(sp, (int)grid, ctx->stream) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return 1;   // nothing was queued: take the launch-per-iteration path
-  }
-  ++ctx->launches;
-  return IDKM_OK;
-}
-
-// The single-launch loop for what try_small_loop does not take: batched layers and single layers beyond its size, with
-// at most 16 centroids.  Returns IDKM_OK after queueing the loop, 1 if this problem should take the
-// launch-per-iteration path.
-static int try_batch_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassParams& p0, int max_iter) {
-  static const bool env_off = (getenv("IDKM_NO_COOP") != nullptr);   // tuning knob: always a launch per iteration
-  if (env_off || (ctx->forward_loop != 0 && ctx->forward_loop != 4) || ctx->squared || ctx->collapse_step != 0 || max_iter < 2) return 1;
-  const LoopEntry* le = loop_entry(ctx->d, ctx->k);
-  if (!le) return 1;
-  // Where the single launch was measured against the launch per iteration (B200, 30 iterations; batches of 21 x 50 K,
-  // 8 x 1 M and a ResNet-18-like mix of rows; both with one resident wave of blocks): it is faster only for 5..8
-  // scalar centroids (22 against 26, 33 against 40, 38 against 43 us per iteration) and for 3..4 centroids at d = 2
-  // (19.5 against 21.8 us on the small batch, level on the large ones); elsewhere the launch per iteration, whose
-  // next launch is scheduled while the epilogue of the last one drains, is level or ahead (d = 4, k = 8, 8 x 1 M: 84
-  // against 128 us -- the joint kernel keeps fewer blocks resident than the fp32 step alone).  Those two classes take
-  // the single launch by default; forward-loop method 4 takes it wherever its kernel exists.
-  if (ctx->forward_loop != 4) {
-    if (ctx->n_layers < 2) return 1;
-    const bool cls_a = (ctx->d == 1 && ctx->k > 4 && ctx->k <= 8), cls_b = (ctx->d == 2 && ctx->k > 2 && ctx->k <= 4);
-    if (!cls_a && !cls_b) return 1;
-  }
-  const int di = d_index(ctx->d), cls = ctx->k <= 2 ? 0 : (ctx->k <= 4 ? 1 : (ctx->k <= 8 ? 2 : 3));
-  int& nb = ctx->loop_blocks[di][cls];
-  if (nb == 0) {
-    int coop = 0, per_sm = 0;
-    nb = -1;
-    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
-        cudaFuncSetAttribute(le->func, cudaFuncAttributeMaxDynamicSharedMemorySize, le->dyn_smem > 0 ? le->dyn_smem : 1) == cudaSuccess &&
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, le->func, BLOCK, le->dyn_smem) == cudaSuccess && per_sm >= 1)
-      nb = ctx->sms * (per_sm > MAX_BLOCKS_PER_SM ? MAX_BLOCKS_PER_SM : per_sm);
-    (void)cudaGetLastError();
-  }
-  if (nb <= 0) return 1;
-  LoopParams lp;
-  memset(&lp, 0, sizeof(lp));
-  lp.p = p0;
-  lp.q = p0;
-  int rc = build_table(ctx, STEP, pick_family(STEP, ctx->d, ctx->k), &lp.p.lt);
-  if (rc != IDKM_OK) return rc;
-  rc = build_table(ctx, STEP_DELTA, pick_family(STEP_DELTA, ctx->d, ctx->k), &lp.q.lt);
-  if (rc != IDKM_OK) return rc;
-  // all blocks are resident at once: each table spreads its tiles over at most that many
-  const int cap = nb;
-  if (lp.p.lt.n_blocks > cap) lp.p.lt.n_blocks = cap;
-  if (lp.q.lt.n_blocks > cap) lp.q.lt.n_blocks = cap;
-  const int grid = lp.p.lt.n_blocks > lp.q.lt.n_blocks ? lp.p.lt.n_blocks : lp.q.lt.n_blocks;
-  char* ws = static_cast<char*>(ctx->workspace);
-  lp.q.partials = reinterpret_cast<double*>(ws + wl.off_partials64);
-  lp.q.gpartials = reinterpret_cast<double*>(ws + wl.off_gpartials64);
-  lp.q.gtickets = reinterpret_cast<unsigned int*>(ws + wl.off_gtickets64);
-  lp.p.host_flag = lp.q.host_flag = nullptr;
-  lp.sync = reinterpret_cast<unsigned int*>(ws + wl.off_sync);
-  lp.max_iter = max_iter;
-  lp.spin_limit = SMALL_SPIN_LIMIT;
-  lp.missing_arrivals = ctx->hook_missing_arrivals;
-  if (ctx->hook_spin_limit > 0 && ctx->hook_spin_limit < SMALL_SPIN_LIMIT) lp.spin_limit = ctx->hook_spin_limit;
-  if (le->launch(lp, grid, ctx->stream) != cudaSuccess) {
     (void)cudaGetLastError();
     return 1;   // nothing was queued: take the launch-per-iteration path
   }
@@ -762,7 +719,6 @@ int idkm_forward_batched(idkm_ctx* ctx, const float* W_cat, const int64_t* layer
 
   nvtxRangePushA("idkm forward loop");
   int rc = try_small_loop(ctx, wl, p, max_iter);
-  if (rc == 1) rc = try_batch_loop(ctx, wl, p, max_iter);
   if (rc == 1) rc = launch_step_loop(ctx, wl, &p, max_iter);
   nvtxRangePop();
   if (rc != IDKM_OK) return rc;
@@ -1085,7 +1041,7 @@ int idkm_set_collapse_step(idkm_ctx* ctx, int method) {
 
 int idkm_set_forward_loop(idkm_ctx* ctx, int method) {
   if (!ctx) return IDKM_ERR_NULL;
-  if (method < 0 || method > 4) return IDKM_ERR_PARAM;
+  if (method < 0 || method > 3) return IDKM_ERR_PARAM;
   ctx->forward_loop = method;
   return IDKM_OK;
 }

@@ -259,13 +259,9 @@ __device__ __forceinline__ double block_sum_double(double v, double* scratch) { 
 // DELTA (forward step of a collapsing layer in the increment form, see delta_body): the totals are
 // dS_j = sum_i (A_ij - 1/k), dN_j = sum_i (A_ij - 1/k) (w_i - c_0) and, in the last D entries, sum_i w_i; with
 // U = sum_i w_i - m c_0 the M-step is C+_j = c_0 + (U / k + dN_j) / (m / k + dS_j).
-// iter_arg: index of the forward iteration when the caller is a loop inside one launch (otherwise the launch's, p.iter).
-constexpr int ITER_OF_LAUNCH = -0x7fffffff;
 template <int MODE, int D, int PLEN, int NA, bool DELTA = false>
-__device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, unsigned char* smem_raw, int* s_flag,
-                                             int iter_arg = ITER_OF_LAUNCH) {
+__device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, unsigned char* smem_raw, int* s_flag) {
   const int tid = threadIdx.x;
-  const int iter = (iter_arg == ITER_OF_LAUNCH) ? p.iter : iter_arg;
   const int k = p.k;
   const int nb = p.lt.n_blocks;
   __threadfence();
@@ -483,7 +479,7 @@ __device__ __forceinline__ void finish_layer(const PassParams& p, int l, int b, 
   if (tid == 0) {
     st->ticket = 0u;
     if constexpr (MODE == STEP) {
-      st->precise[(iter + 1) & 1] = (!p.squared && sqrt(box2) * p.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
+      st->precise[(p.iter + 1) & 1] = (!p.squared && sqrt(box2) * p.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
       double dn = sqrt(den);
       if (dn < 1e-300) dn = 1e-300;
       const float res = (float)(sqrt(num) / dn);
@@ -622,10 +618,8 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, unsign
 // asynchronous copy per trip (cp.async.bulk, completion on an mbarrier), issued by one thread BULK_STAGES trips ahead
 // of the arithmetic, instead of by per-thread 128-bit loads issued at the top of the trip.
 template <int MODE, int D, int KPL, int LPW, bool RELEASE, bool SQ = false, bool BULK = false>
-__device__ __forceinline__ void pass_body(const PassParams& p, int iter_arg = ITER_OF_LAUNCH) {
+__device__ __forceinline__ void pass_body(const PassParams& p) {
   using Cfg = PassCfg<MODE, D, KPL, LPW>;
-  const int iter = (iter_arg == ITER_OF_LAUNCH) ? p.iter : iter_arg;   // forward iteration this call steps
-  (void)iter;
   constexpr int NACC = Cfg::NACC;
   constexpr int PLEN = Cfg::PLEN;
   constexpr int WPG = Cfg::WPG;
@@ -977,7 +971,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p, int iter_arg = IT
         for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv * PLEN + o];
         mine[o] = s;
       }
-      finish_layer<MODE, D, PLEN, NA>(p, l, b, smem_raw, &s_flag, iter);
+      finish_layer<MODE, D, PLEN, NA>(p, l, b, smem_raw, &s_flag);
     }
   };
 
@@ -1044,8 +1038,8 @@ __device__ __forceinline__ void pass_body(const PassParams& p, int iter_arg = IT
         const int a = (lim - ptile < Cfg::UNROLL) ? lim - ptile : Cfg::UNROLL;
         const int tl = ptile;
         ptile += a;
-        const bool act = (p.st[player].fwd_done == 0) && (p.st[player].precise[iter & 1] == 0) &&
-                         (p.st[player].fwd_iters == iter);
+        const bool act = (p.st[player].fwd_done == 0) && (p.st[player].precise[p.iter & 1] == 0) &&
+                         (p.st[player].fwd_iters == p.iter);
         const long long r0 = p.lt.row_off[player];
         if (!act || (r0 * D) % 4 != 0) continue;
         const long long rws = p.lt.row_off[player + 1] - r0;
@@ -1088,7 +1082,7 @@ __device__ __forceinline__ void pass_body(const PassParams& p, int iter_arg = IT
       if (cur_layer >= 0 && layer_active) flush(cur_layer);
       cur_layer = layer;
       if constexpr (MODE == STEP)
-        layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[iter & 1] == 0) && (p.st[layer].fwd_iters == iter);
+        layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[p.iter & 1] == 0) && (p.st[layer].fwd_iters == p.iter);
       else if constexpr (MODE == ADJ) layer_active = (p.st[layer].adj_done == 0);
       else layer_active = true;
       if constexpr (US_SMEM) __syncthreads();   // the previous layer's table is no longer read
@@ -1649,10 +1643,9 @@ __device__ __forceinline__ float expm1_small(float x) {
   return fmaf(s * x, x, x);
 }
 
-template <int D, int KPL, int LPW, bool RELEASE = true>
-__device__ __forceinline__ void delta_body(const PassParams& p, int iter_arg = ITER_OF_LAUNCH) {
+template <int D, int KPL, int LPW>
+__device__ __forceinline__ void delta_body(const PassParams& p) {
   using Cfg = DeltaCfg<D, KPL, LPW>;
-  const int iter = (iter_arg == ITER_OF_LAUNCH) ? p.iter : iter_arg;
   constexpr int NA = Cfg::NA, PLEN = Cfg::PLEN, PLENK = Cfg::PLENK, WPG = Cfg::WPG, TILE = Cfg::TILE, NSLOT = Cfg::NSLOT;
   constexpr int NEXTRA = Cfg::NEXTRA;
   constexpr int RED_BYTES = NWARP * PLEN * 4;
@@ -1756,7 +1749,7 @@ __device__ __forceinline__ void delta_body(const PassParams& p, int iter_arg = I
       for (int wv = 0; wv < NWARP; ++wv) sres += (double)red[wv * PLEN + o];
       mine[o] = sres;
     }
-    finish_layer<STEP, D, PLEN, NA, true>(p, l, b, smem_raw, &s_flag, iter);
+    finish_layer<STEP, D, PLEN, NA, true>(p, l, b, smem_raw, &s_flag);
   };
 
   // full_tag: the codebook fills every centroid slot of the layout (no per-centroid validity tests)
@@ -1848,7 +1841,7 @@ __device__ __forceinline__ void delta_body(const PassParams& p, int iter_arg = I
     if (layer != cur_layer) {
       if (cur_layer >= 0 && layer_active) flush(cur_layer);
       cur_layer = layer;
-      layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[iter & 1] != 0) && (p.st[layer].fwd_iters == iter);
+      layer_active = (p.st[layer].fwd_done == 0) && (p.st[layer].precise[p.iter & 1] != 0) && (p.st[layer].fwd_iters == p.iter);
       if (layer_active) {
         const float* Cl = p.C + (size_t)layer * k * D;
         inv_k = 1.f / (float)k;
@@ -2003,7 +1996,7 @@ __device__ __forceinline__ void delta_body(const PassParams& p, int iter_arg = I
       since_spill = 0;
     }
   }
-  if constexpr (RELEASE) grid_release_dependents();
+  grid_release_dependents();
   if (cur_layer >= 0 && layer_active) flush(cur_layer);
 }
 
@@ -2012,32 +2005,6 @@ __global__ void __launch_bounds__(BLOCK, DeltaCfg<D, KPL, LPW>::MIN_BLOCKS)
 idkm_step_delta(const __grid_constant__ PassParams p) {
   grid_dependency_sync();
   delta_body<D, KPL, LPW>(p);
-}
-
-// Grid-wide barrier of a cooperative launch: one arrival counter that only grows (sync[0]) and an error word (sync[1]).
-// Bounded wait until the arrival counter has reached `target`.  Returns false if the wait ran out or another block
-// raised the error word.
-__device__ __forceinline__ bool small_barrier(unsigned int* sync, unsigned int target, long long spin_limit, int* s_ok) {
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    volatile unsigned int* vs = sync;
-    int ok = 1;
-    __threadfence();
-    atomicAdd(&sync[0], 1u);
-    const long long t0 = clock64();
-    while ((int)(vs[0] - target) < 0) {
-      if (vs[1] != 0u || clock64() - t0 > spin_limit) {
-        atomicExch(&sync[1], 1u);
-        ok = 0;
-        break;
-      }
-    }
-    if (vs[1] != 0u) ok = 0;
-    __threadfence();
-    *s_ok = ok;
-  }
-  __syncthreads();
-  return *s_ok != 0;
 }
 
 // One launch per forward iteration instead of two, for the smallest thread-per-weight layouts, where the fp32 and
@@ -2061,61 +2028,6 @@ idkm_step_dual(const __grid_constant__ DualParams dp) {
 }
 
 
-// The whole forward loop (Algorithm 1) of a BATCH of layers, or of one layer too large for idkm_small_loop, in ONE
-// cooperative launch: per iteration every block runs the fp32 step on its tiles of the layers that have not collapsed
-// and the increment-form step on its tiles of those that have -- the very bodies (tile tables, partial slots, ticketed
-// two-stage sums, M-step by the last arrival) of the launch-per-iteration kernels -- and then waits at a grid-wide
-// barrier, after which the centroids, flags and counts the epilogues wrote are visible to all.  What a launch per
-// iteration costs beyond the arithmetic (scheduling a grid, refilling the SMs, draining them) is paid once.  The loop
-// ends after max_iter iterations, or at the first barrier at which every layer's loop has ended: a layer that ended
-// with iteration t carries fwd_done = t + 1, which no block can mistake for the outcome of an iteration it has not
-// reached itself, so all blocks leave at the same barrier.  Every barrier wait is bounded; if one runs out the blocks
-// return and block 0 marks the layers ST_TIMEOUT.
-struct LoopParams {
-  PassParams p;            // fp32 step
-  PassParams q;            // increment-form step (own tile table and partial buffers)
-  unsigned int* sync;      // [0] barrier arrivals, [1] error word; both zero before the launch
-  long long spin_limit;    // clock64() ticks a block waits at a barrier before it gives up
-  int missing_arrivals;    // 0 in production (host-side fault injection for the timeout path, see idkm.h)
-  int max_iter;
-};
-template <int D, int KPL, int LPW, int KPLQ, int LPWQ>
-struct LoopCfg {
-  using A = PassCfg<STEP, D, KPL, LPW>;
-  using B = DeltaCfg<D, KPLQ, LPWQ>;
-  static constexpr int MIN_BLOCKS = A::MIN_BLOCKS < B::MIN_BLOCKS ? A::MIN_BLOCKS : B::MIN_BLOCKS;
-  static constexpr int DYN_SMEM = A::DYN_SMEM > B::DYN_SMEM ? A::DYN_SMEM : B::DYN_SMEM;
-};
-template <int D, int KPL, int LPW, int KPLQ, int LPWQ>
-__global__ void __launch_bounds__(BLOCK, LoopCfg<D, KPL, LPW, KPLQ, LPWQ>::MIN_BLOCKS)
-idkm_step_loop(const __grid_constant__ LoopParams lp) {
-  __shared__ int s_ok;
-  const int n_layers = lp.p.lt.n_layers;
-  const unsigned int arrivals = gridDim.x + (unsigned int)lp.missing_arrivals;
-  for (int it = 0; it < lp.max_iter; ++it) {
-    pass_body<STEP, D, KPL, LPW, false>(lp.p, it);
-    __syncthreads();
-    delta_body<D, KPLQ, LPWQ, false>(lp.q, it);
-    if (!small_barrier(lp.sync, (unsigned int)(it + 1) * arrivals, lp.spin_limit, &s_ok)) {
-      if (blockIdx.x == 0)
-        for (int l = threadIdx.x; l < n_layers; l += BLOCK) lp.p.st[l].status = ST_TIMEOUT;
-      return;
-    }
-    // has every layer's loop ended by iteration `it`?  (0 < fwd_done <= it + 1; later outcomes do not count yet)
-    int ended = 1;
-    for (int l = threadIdx.x; l < n_layers; l += BLOCK) {
-      const int fd = *reinterpret_cast<const volatile int*>(&lp.p.st[l].fwd_done);
-      if (fd == 0 || fd > it + 1) ended = 0;
-    }
-    if (__syncthreads_and(ended)) break;
-  }
-}
-typedef cudaError_t (*LoopLaunchFn)(const LoopParams& lp, int grid, cudaStream_t stream);
-struct LoopEntry {
-  LoopLaunchFn launch;
-  const void* func;
-  int dyn_smem;
-};
 
 // Exact solve of (I - J^T) u = g -- the linear system behind M* = (I - dF/dC)^-1 of Section 4.2, contracted with g --
 // by ONE warp: the matrix J (n x n, row stride ld, fp64, shared memory) is turned into I - J^T in place, then Gaussian
@@ -2494,20 +2406,22 @@ struct DualEntry {
   const void* func;
   int dyn_smem;
 };
-// Single-launch forward loop for one small layer (idkm_small_loop.cu): k <= 2, 4, 8, 16 centroids per thread.
+// Single-launch forward loop for small layers (idkm_small_loop.cu): k <= 2, 4, 8, 16 centroids per thread.
 struct SmallLoopParams {
   const float* W;
-  long long m;
-  float* C;              // [k][d]: starting centroids in, returned centroids out
-  LayerState* st;        // the layer's state: `precise` is read at the start, the outcome written at the end
-  double* partials;      // [2][grid][k_pad (d+1)] fp64 block partials, alternating by iteration
+  int n_layers;
+  long long row_off[MAX_LAYERS + 1];   // first row of each layer
+  int blk_first[MAX_LAYERS + 1];       // first block of each layer; blk_first[n_layers] = grid size
+  float* C;              // [L][k][d]: starting centroids in, returned centroids out
+  LayerState* st;        // [L] layer states: `precise` is read at the start, the outcome written at the end
+  double* partials;      // [2][grid][k_pad (d+1) + d] fp64 block partials, alternating by iteration
   unsigned int* sync;    // [0] barrier arrivals (only grows), [1] error word; both zero before the launch
   int k;
   float scale;           // log2(e) / tau
   float tol;
   double inv_tau_d;
   int max_iter;
-  float* hist;           // [HIST_CAP] residual history of the layer
+  float* hist;           // [L][HIST_CAP] residual histories
   int chunked;           // 1: some thread has more than 32 rows, fp32 sums are moved out every 32 rows
   int missing_arrivals;  // 0 in production.  Host-side fault injection for the timeout path: the barriers wait for
                          // this many arrivals more than the grid has, so every wait runs out (see idkm.h)

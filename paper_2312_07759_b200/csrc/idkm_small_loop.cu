@@ -1,4 +1,6 @@
-// Algorithm 1's whole loop in ONE cooperative launch, for a single small layer (k <= 16, a few million weights at most).
+// Algorithm 1's whole loop in ONE cooperative launch, for a small layer or a batch of layers (k <= 16, a few million
+// weights per layer at most).  Every block works for exactly one layer: the layers share the grid in proportion to their
+// rows (at least one block each) and the grid-wide barrier; everything else below happens per layer, among its blocks.
 //
 // There one iteration is a few microseconds of arithmetic, and a launch per iteration -- with its chain of dependent
 // trips to L2 (partials, ticket, totals, centroids, state) -- costs more than the arithmetic.  Here all blocks are
@@ -17,11 +19,40 @@ template <int D, int KPL>
 struct SmallCfg {
   static constexpr int NA = D + 1;
   static constexpr int PLENK = KPL * NA;           // per-centroid sums
-  static constexpr int PLEN = PLENK + D;           // ... and the sum of the weights (increment-form iterations)
+  // ... then, for increment-form iterations, the sum of the weights and (scalar weights) count and sum of the rows
+  // above / below all centroids, which need no per-centroid work
+  static constexpr int NEXTRA = (D == 1) ? 4 : 0;
+  static constexpr int PLEN = PLENK + D + NEXTRA;
   static constexpr int CH = BLOCK / PLEN;          // chunks of partial rows added in parallel in the second level
   static constexpr int KD = KPL * D;
   static constexpr int DYN_SMEM = PLEN * BLOCK * 4;
 };
+
+// Grid-wide barrier of a cooperative launch: one arrival counter that only grows (sync[0]) and an error word (sync[1]).
+// Bounded wait until the arrival counter has reached `target`.  Returns false if the wait ran out or another block
+// raised the error word.
+__device__ __forceinline__ bool small_barrier(unsigned int* sync, unsigned int target, long long spin_limit, int* s_ok) {
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    volatile unsigned int* vs = sync;
+    int ok = 1;
+    __threadfence();
+    atomicAdd(&sync[0], 1u);
+    const long long t0 = clock64();
+    while ((int)(vs[0] - target) < 0) {
+      if (vs[1] != 0u || clock64() - t0 > spin_limit) {
+        atomicExch(&sync[1], 1u);
+        ok = 0;
+        break;
+      }
+    }
+    if (vs[1] != 0u) ok = 0;
+    __threadfence();
+    *s_ok = ok;
+  }
+  __syncthreads();
+  return *s_ok != 0;
+}
 
 // CHUNKED: some thread has more than SMALL_CHUNK rows; its fp32 sums are then moved out every SMALL_CHUNK rows.
 template <int D, int KPL, bool CHUNKED>
@@ -37,15 +68,23 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
   extern __shared__ __align__(16) float slots[];   // [PLEN][BLOCK] second-level fp32 sums (CHUNKED only)
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.x, G = gridDim.x;
+  const int G = gridDim.x;
   const int k = sp.k;
-  const long long m = sp.m;
+  // this block's layer, its rank among the layer's blocks (b) and their number (NB)
+  int layer = 0;
+  while (layer + 1 < sp.n_layers && (int)blockIdx.x >= sp.blk_first[layer + 1]) ++layer;
+  const int first_blk = sp.blk_first[layer];
+  const int b = (int)blockIdx.x - first_blk, NB = sp.blk_first[layer + 1] - first_blk;
+  const long long m = sp.row_off[layer + 1] - sp.row_off[layer];
+  const float* Wl = sp.W + sp.row_off[layer] * D;
+  float* Cl = sp.C + (size_t)layer * k * D;
+  LayerState* st = sp.st + layer;
 
-  // uniform loop state (identical in every thread of every block)
+  // uniform loop state (identical in every thread of every block of the layer)
   int iters = 0, done = 0, status = ST_OK, dead_n = 0;
-  int precise = sp.st[0].precise[0];
+  int precise = st->precise[0];
   float res_f = 0.f;
-  if (tid < k * D) c_sm[tid] = sp.C[tid];
+  if (tid < k * D) c_sm[tid] = Cl[tid];
   __syncthreads();
   float c[KPL][D];
 #pragma unroll
@@ -56,20 +95,22 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
   const float inv_k = 1.f / (float)k;
   bool ok = true;
 
-  for (int it = 0; it < sp.max_iter && !done; ++it) {
+  for (int it = 0; it < sp.max_iter; ++it) {
+    if (sp.n_layers == 1 && done) break;   // (a batch goes on meeting at the barrier until every layer has ended)
     // ---- this block's rows and its partial (fixed order: lanes by shuffle tree, warps in index order) ----
-    double* mine = sp.partials + ((size_t)(it & 1) * G + b) * PLEN;
+    double* mine = sp.partials + ((size_t)(it & 1) * G + blockIdx.x) * PLEN;
     auto load_row = [&](long long r, float (&w)[D]) {
       if constexpr (D == 4) {
-        const float4 x = __ldg(reinterpret_cast<const float4*>(sp.W) + r);
+        const float4 x = __ldg(reinterpret_cast<const float4*>(Wl) + r);
         w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
       } else if constexpr (D == 2) {
-        const float2 x = __ldg(reinterpret_cast<const float2*>(sp.W) + r);
+        const float2 x = __ldg(reinterpret_cast<const float2*>(Wl) + r);
         w[0] = x.x; w[1] = x.y;
       } else {
-        w[0] = __ldg(sp.W + r);
+        w[0] = __ldg(Wl + r);
       }
     };
+    if (!done) {
     // Sums of this thread: [t * NA + a] per centroid, then D entries for the sum of the weights (increment form only).
     // A long fp32 running sum drops the many terms below half its ulp (one-sided): threads with more than
     // SMALL_CHUNK rows move their sums into a private shared-memory slot every SMALL_CHUNK rows.
@@ -91,11 +132,11 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
     // processed; what does not fill a 128-bit load (and everything, if W is not 16-byte aligned) by row.
     auto walk = [&](auto&& row) {
       constexpr int VEC = 4 / D;
-      const long long stride = (long long)G * BLOCK;
+      const long long stride = (long long)NB * BLOCK;
       long long first_by_row = 0;
-      if ((reinterpret_cast<size_t>(sp.W) & 15) == 0) {
+      if ((reinterpret_cast<size_t>(Wl) & 15) == 0) {
         const long long nvec = m / VEC;
-        const float4* W4 = reinterpret_cast<const float4*>(sp.W);
+        const float4* W4 = reinterpret_cast<const float4*>(Wl);
         long long q = (long long)b * BLOCK + tid;
         float4 cur = make_float4(0.f, 0.f, 0.f, 0.f), n1 = cur, n2 = cur;
         if (q < nvec) cur = __ldg(W4 + q);
@@ -187,10 +228,27 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
         }
         dl2[t] = (float)d2;
       }
+      // scalar weights: a row farther than twice the largest |delta_j| from c_0 lies outside all centroids; its
+      // attention increments take one of two values per centroid (applied in the M-step), so it is only counted
+      float dmax2 = 0.f;
+      if constexpr (D == 1) {
+#pragma unroll
+        for (int t = 0; t < KPL; ++t) dmax2 = fmaxf(dmax2, 2.f * fabsf(dl[t][0]));
+      }
       walk([&](const float (&w)[D]) {
         float u[D], x[KPL];
 #pragma unroll
         for (int a = 0; a < D; ++a) u[a] = w[a] - c0[a];
+        if constexpr (D == 1) {
+          if (fabsf(u[0]) > dmax2) {
+            const bool pos = (u[0] > 0.f);
+            sum[PLENK + 1] += pos ? 1.f : 0.f;
+            sum[PLENK + 2] += pos ? w[0] : 0.f;
+            sum[PLENK + 3] += pos ? 0.f : 1.f;
+            sum[PLENK + 4] += pos ? 0.f : w[0];
+            return;
+          }
+        }
         if constexpr (D == 1) {
           // |u - delta| - |u| without forming u - delta: with s = sign(u), -s delta + 2 max(0, s delta - |u|)
           const float aut = fabsf(u[0]) * inv_tau;
@@ -252,16 +310,29 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
       __stcg(mine + tid, s);
     }
+    }   // !done
     // ---- everyone has published: grid-wide barrier ----
     ok = small_barrier(sp.sync, (unsigned int)(it + 1) * (unsigned int)(G + sp.missing_arrivals), sp.spin_limit, &s_ok);
     if (!ok) break;
-    // ---- every block adds all partials in the same order ----
+    // A batch ends at the first barrier at which every layer's loop has ended: the first block of a layer publishes
+    // fwd_done = (iterations taken) before it arrives at the next barrier, so after barrier `it` every value in
+    // (0, it] is final and seen by all blocks alike; a later value cannot be mistaken for one of them.
+    if (sp.n_layers > 1 && sp.tol > 0.f) {
+      int ended = 1;
+      for (int l = tid; l < sp.n_layers; l += BLOCK) {
+        const int fd = *reinterpret_cast<const volatile int*>(&sp.st[l].fwd_done);
+        if (fd == 0 || fd > it) ended = 0;
+      }
+      if (__syncthreads_and(ended)) break;
+    }
+    if (done) continue;
+    // ---- every block of the layer adds the layer's partials in the same order ----
     {
-      const double* base = sp.partials + (size_t)(it & 1) * G * PLEN;
+      const double* base = sp.partials + ((size_t)(it & 1) * G + first_blk) * PLEN;
       const int ch = tid / PLEN, o = tid % PLEN;
       if (ch < CH) {
         double s = 0.0;
-        for (int q = ch; q < G; q += CH) s += __ldcg(base + (size_t)q * PLEN + o);
+        for (int q = ch; q < NB; q += CH) s += __ldcg(base + (size_t)q * PLEN + o);
         chunk[ch][o] = s;
       }
       __syncthreads();
@@ -281,14 +352,36 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       double num = 0.0, den = 0.0, bad = 0.0, dead = 0.0, cq = 0.0;
       // increment form: centroid 0 as it was when the rows were taken (read by all lanes before any lane writes)
       const double c0a = (double)c_sm[own ? a : 0];
+      double tS = own ? tot[j * NA] : 0.0, tN = own ? tot[j * NA + 1 + a] : 0.0, wsum = own ? tot[PLENK + a] : 0.0;
+      if constexpr (D == 1) {
+        if (precise) {
+          // the rows that were only counted: above all centroids their logit differences are +delta_j / tau, below
+          // -delta_j / tau, whatever their own value
+          const double cp = tot[PLENK + 1], sp_ = tot[PLENK + 2], cm = tot[PLENK + 3], sm = tot[PLENK + 4];
+          const double dj = own ? ((double)c_sm[lane] - c0a) * sp.inv_tau_d : 0.0;
+          const double tpj = own ? expm1(dj) : 0.0, tmj = own ? expm1(-dj) : 0.0;
+          double tbp = tpj, tbm = tmj;
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            tbp += __shfl_xor_sync(0xffffffffu, tbp, o);
+            tbm += __shfl_xor_sync(0xffffffffu, tbm, o);
+          }
+          tbp /= (double)k;
+          tbm /= (double)k;
+          const double ap = (tpj - tbp) / ((double)k * (1.0 + tbp)), am = (tmj - tbm) / ((double)k * (1.0 + tbm));
+          tS += ap * cp + am * cm;
+          tN += ap * (sp_ - cp * c0a) + am * (sm - cm * c0a);
+          wsum += sp_ + sm;
+        }
+      }
       __syncwarp();
       if (own) {
         const double mk = (double)m / (double)k;
-        const double s = precise ? mk + tot[j * NA] : tot[j * NA];
+        const double s = precise ? mk + tS : tS;
         const bool alive = (s >= S_MIN);
         const double cold = (double)c_sm[lane];
-        const double ubar = precise ? (tot[PLENK + a] - (double)m * c0a) / (double)k : 0.0;
-        const double cnew = alive ? (precise ? c0a + (ubar + tot[j * NA + 1 + a]) / s : tot[j * NA + 1 + a] / s) : cold;
+        const double ubar = precise ? (wsum - (double)m * c0a) / (double)k : 0.0;
+        const double cnew = alive ? (precise ? c0a + (ubar + tN) / s : tN / s) : cold;
         if (!alive && a == 0) dead = 1.0;
         if (!(s == s) || s > 1e300 || !(cnew == cnew) || fabs(cnew) > 1e300) bad = 1.0;
         num = (cnew - cold) * (cnew - cold);
@@ -329,25 +422,25 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       for (int a = 0; a < D; ++a) c[t][a] = (t < k) ? c_sm[t * D + a] : PAD_COORD;
     iters = it + 1;
     res_f = (float)s_res[0];
-    if (b == 0 && tid == 0 && iters <= HIST_CAP) sp.hist[iters - 1] = res_f;
+    if (b == 0 && tid == 0 && iters <= HIST_CAP) sp.hist[(size_t)layer * HIST_CAP + iters - 1] = res_f;
     dead_n = (int)s_res[1];
     precise = (sqrt(s_res[3]) * sp.inv_tau_d <= PRECISE_SPAN) ? 1 : 0;
     if (s_res[2] > 0.0) {
       status = ST_NONFINITE;
-      done = 1;
+      done = iters;
     } else if (sp.tol > 0.f && res_f < sp.tol) {
-      done = 1;
+      done = iters;
       status = ST_OK;
     } else if (sp.tol > 0.f && iters >= sp.max_iter) {
       status = ST_MAXITER;
     }
+    if (done && b == 0 && tid == 0) st->fwd_done = done;   // (seen by the other layers' blocks after the next barrier)
     __syncthreads();
   }
 
   if (b == 0) {
-    if (tid < k * D) sp.C[tid] = c_sm[tid];
+    if (tid < k * D) Cl[tid] = c_sm[tid];
     if (tid == 0) {
-      LayerState* st = sp.st;
       st->fwd_iters = iters;
       st->fwd_res = res_f;
       st->dead = dead_n;
