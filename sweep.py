@@ -42,7 +42,13 @@ def run_point(ctx, B, torch, m, d, b, tau, cap):
     dev = torch.device("cuda", 0)
     W, C0, G = (torch.from_numpy(x).to(dev) for x in (wl.W, wl.C0, wl.G))
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
-    ctx.forward(W, C0, wl.tau, wl.tol, 3)                      # warm-up (kernel load, caches)
+    # warm-up: every kernel the timed calls use is launched once before (the first launch of a kernel loads it, which
+    # takes up to a millisecond and would otherwise land in the first point of each (d, k))
+    ctx.forward(W, C0, wl.tau, wl.tol, 3)
+    ctx.forward(W, C0, wl.tau, 0.0, 3)
+    ctx.backward(G, B.JFB, 0.0, 0, 1.0)
+    ctx.backward(G, B.IMPLICIT, wl.adj_tol, 3, 1.0)
+    ctx.backward(G, B.IMPLICIT, 0.0, 20, 1.0)
     torch.cuda.synchronize()
     ev[0].record()
     ctx.forward(W, C0, wl.tau, wl.tol, cap)
@@ -55,11 +61,14 @@ def run_point(ctx, B, torch, m, d, b, tau, cap):
     info = ctx.info()[0]
     # the same number of iterations at a fixed count: the time of the executed iterations alone (launches queued
     # after convergence return at once but still cost a few microseconds each)
-    ev[4].record()
-    ctx.forward(W, C0, wl.tau, 0.0, max(info.fwd_iters, 1))
-    ev[5].record()
-    torch.cuda.synchronize()
-    fixed_ms = ev[4].elapsed_time(ev[5])
+    # (timed by the library's own events around the loop, second of two calls: an event pair around the call would
+    # also count the host's allocation of the call's outputs, which stalls the stream when a new size appears)
+    ctx.set_timing(True)
+    for _ in range(2):
+        ctx.forward(W, C0, wl.tau, 0.0, max(info.fwd_iters, 1))
+        torch.cuda.synchronize()
+    fixed_ms = ctx.phase_ms()["steps"]
+    ctx.set_timing(False)
     ctx.forward(W, C0, wl.tau, wl.tol, cap)                    # restore the tolerance-mode state for the reference
     dWr, dCr = ctx.backward(G, B.IMPLICIT, 0.0, 200, 1.0)     # the 200-iteration reference
     torch.cuda.synchronize()
