@@ -86,3 +86,42 @@ def test_barrier_timeout_is_reported_and_the_context_survives():
     again = ctx.forward(W, C0, wl.tau, 0.0, 6).C.cpu().numpy()
     assert ctx.info()[0].status == 0 and ctx.info()[0].fwd_iters == 6
     assert np.array_equal(again, good)
+
+
+@pytest.mark.parametrize("d,k", [(1, 4), (2, 8), (4, 4), (4, 16)])
+def test_guard_words_around_a_batched_call(d, k):
+    """The same for a batch of five layers (ragged sizes, a layer of one block, unaligned layer starts), on the
+    one-launch loop and on the launch-per-iteration path, forward and both backward modes."""
+    import ctypes
+    import torch
+    from paper_2312_07759_b200 import binding as B
+    ms = [70001, 3000, 40000, 517, 131072]
+    parts = [WL.single_layer(m, d, k, 0.004, std=0.02 + 0.01 * i, seed=31 + i) for i, m in enumerate(ms)]
+    W = np.concatenate([p_.W for p_ in parts])
+    C0 = np.concatenate([p_.C0 for p_ in parts])
+    G = np.concatenate([p_.G for p_ in parts])
+    L, m = len(ms), int(sum(ms))
+    offs_host = (ctypes.c_int64 * (L + 1))(*np.concatenate([[0], np.cumsum(ms)]).tolist())
+    ws_bytes = B.workspace_bytes(m, d, k, L)
+    sizes = [4 * L * k * d, 4 * m * d, 4 * m * d, 4 * L * k * d, ws_bytes]       # C, Wq, dW, dC, workspace
+    buf, offs = _carve(torch, sizes)
+    p = [buf.data_ptr() + o for o in offs]
+    Wd, C0d, Gd = (torch.from_numpy(x).cuda() for x in (W, C0, G))
+    results = []
+    for loop_method in (0, 1):
+        ctx = B.Context()
+        ctx.set_forward_loop(loop_method)
+        rc = B.lib.idkm_forward_batched(ctx._h, Wd.data_ptr(), offs_host, L, d, C0d.data_ptr(), k, 0.004, 0.0, 7,
+                                        p[0], None, p[1], p[4], ws_bytes, None)
+        assert rc == 0
+        assert ctx.backward_raw(Gd.data_ptr(), B.JFB, 0.0, 0, 1.0, p[2], p[3], p[4], ws_bytes) == 0
+        assert ctx.backward_raw(Gd.data_ptr(), B.IMPLICIT, 0.0, 20, 1.0, p[2], p[3], p[4], ws_bytes) == 0
+        torch.cuda.synchronize()
+        ctx.n_layers = L
+        # (seven iterations do not reach a fixed point, where the adjoint iteration need not contract: that status is
+        # legitimate here)
+        infos = ctx.info()
+        assert all(i.status in (0, B.ERR_DIVERGED) and i.fwd_iters == 7 for i in infos), infos
+        _check(torch, buf, offs, sizes)
+        results.append(buf[offs[0]:offs[0] + sizes[0]].clone().view(torch.float32).cpu().numpy())
+    assert np.abs(results[0] - results[1]).max() <= 2e-6 * np.abs(results[1]).max()
