@@ -472,12 +472,14 @@ static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams
 // The single-launch loop of idkm_small_loop.cu takes layers with k <= 16 (k <= 8 for d = 4): a single layer whose rows
 // fit SMALL_ROWS_PER_THREAD per thread of the co-resident grid -- about 4.8 million rows on a 148-SM part (beyond that
 // the tiled step kernels with their deeper load pipelines are as fast) -- or a batch of up to as many layers as the grid
-// has blocks, with up to SMALL_BATCH_ROWS_PER_THREAD rows per thread (a batch pays more per iteration on the tiled path:
-// every block there walks several layers, each with its own chain of block sums and tickets).  The blocks are dealt out
+// has blocks, with up to SMALL_BATCH_ROWS_PER_THREAD rows per thread and SMALL_BATCH_MAX_FLOATS weights in all (a batch
+// pays more per iteration on the tiled path: every block there walks several layers, each with its own chain of block
+// sums and tickets).  The blocks are dealt out
 // to the layers in proportion to their rows, at least one each, and at least SMALL_MIN_ROWS_PER_THREAD rows per thread:
 // tiny layers use few blocks, which keeps the cross-block sum short.
 constexpr int SMALL_ROWS_PER_THREAD = 64;
 constexpr int SMALL_BATCH_ROWS_PER_THREAD = 256;
+constexpr long long SMALL_BATCH_MAX_FLOATS = 20LL << 20;   // 80 MB of weights: they stay in the 126 MB L2 across iterations
 constexpr int SMALL_CHUNK_ROWS = 32;   // threads with more rows than this move their fp32 sums out every 32 rows
 constexpr int SMALL_MIN_ROWS_PER_THREAD = 4;
 constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM clock ticks per barrier wait
@@ -508,8 +510,10 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   const int L = ctx->n_layers;
   const long long m = ctx->m_total;
   if (L > nb || L > MAX_LAYERS) return 1;
-  // (d = 4 batches beyond the single-layer size measured slower than a launch per iteration: 8 x 1 M rows, 65 against 41 us)
-  if (m > (long long)((L == 1 || ctx->d == 4) ? SMALL_ROWS_PER_THREAD : SMALL_BATCH_ROWS_PER_THREAD) * nb * BLOCK) return 1;
+  if (m > (long long)(L == 1 ? SMALL_ROWS_PER_THREAD : SMALL_BATCH_ROWS_PER_THREAD) * nb * BLOCK) return 1;
+  // (a batch whose weights do not stay in L2 is faster by a launch per iteration, whose kernels keep more loads in
+  // flight: 16 x 1 M rows at d = 2, k = 2: 68 against 38 us per iteration; 8 x 1 M at d = 4, k = 2: 65 against 41 us)
+  if (L > 1 && m * ctx->d > SMALL_BATCH_MAX_FLOATS) return 1;
   long long grid = (m + (long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK - 1) / ((long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK);
   if (grid > nb) grid = nb;
   if (grid < L) grid = L;
