@@ -309,10 +309,10 @@ int idkm_measure_pipe_rates(double* fp32_lane_ops_per_s, double* sfu_lane_ops_pe
 
 /*
  * How the forward loop (Algorithm 1) is launched.  0 (default): layers with k <= 16 (k <= 8 for d = 4) run the WHOLE
- * loop in one cooperative launch -- a single layer of at most about 4.8 million rows (64 rows per thread of the
- * co-resident grid), or a batch of layers (Algorithm 2 clusters every layer of the network before each minibatch:
- * "for all layers") of at most four times that in total, at most 80 MB of weights (they then stay in L2 across the
- * iterations) and no more layers than the grid has blocks.  The blocks are dealt out to the layers in proportion to their rows, at least one each; per
+ * loop in one cooperative launch -- a single layer of at most about 9.7 million rows (128 rows per thread of the
+ * co-resident grid; half that at d = 4), or a batch of layers (Algorithm 2 clusters every layer of the network before
+ * each minibatch: "for all layers") of at most twice that in total and no more layers than the grid has blocks;
+ * either way at most 80 MB of weights (they then stay in L2 across the iterations).  The blocks are dealt out to the layers in proportion to their rows, at least one each; per
  * iteration every block publishes one fp64 partial of its layer, all blocks meet at a grid-wide barrier, and every
  * block then adds its layer's partials in the same order and takes the M-step itself, so only the partials cross L2
  * inside the loop.  A layer leaves the loop at the iteration whose stop test passes; a batch leaves at the first

@@ -470,16 +470,18 @@ static int launch_step_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, PassParams
 }
 
 // The single-launch loop of idkm_small_loop.cu takes layers with k <= 16 (k <= 8 for d = 4): a single layer whose rows
-// fit SMALL_ROWS_PER_THREAD per thread of the co-resident grid -- about 4.8 million rows on a 148-SM part (beyond that
-// the tiled step kernels with their deeper load pipelines are as fast) -- or a batch of up to as many layers as the grid
-// has blocks, with up to SMALL_BATCH_ROWS_PER_THREAD rows per thread and SMALL_BATCH_MAX_FLOATS weights in all (a batch
-// pays more per iteration on the tiled path: every block there walks several layers, each with its own chain of block
-// sums and tickets).  The blocks are dealt out
+// fit SMALL_ROWS_PER_THREAD per thread of the co-resident grid -- about 9.7 million rows on a 148-SM part, 4.8 million at
+// d = 4 (measured against a launch per iteration at m = 5 .. 9.5 million: 11.6 against 17.4 us at d = 1, k = 2, m = 5 M;
+// 22.8 against 24.4 us at d = 1, k = 4, m = 9.5 M; d = 4, k = 8, collapsing, m = 5 M: 85 against 66 us, hence the lower
+// limit there) -- or a batch of up to as many layers as the grid has blocks, with up to SMALL_BATCH_ROWS_PER_THREAD rows
+// per thread; either way at most SMALL_MAX_FLOATS weights in all (a batch pays more per iteration on the tiled path:
+// every block there walks several layers, each with its own chain of block sums and tickets).  The blocks are dealt out
 // to the layers in proportion to their rows, at least one each, and at least SMALL_MIN_ROWS_PER_THREAD rows per thread:
 // tiny layers use few blocks, which keeps the cross-block sum short.
-constexpr int SMALL_ROWS_PER_THREAD = 64;
+constexpr int SMALL_ROWS_PER_THREAD = 128;      // a single layer, d <= 2
+constexpr int SMALL_ROWS_PER_THREAD_D4 = 64;    // a single layer, d = 4 (one row per 128-bit load)
 constexpr int SMALL_BATCH_ROWS_PER_THREAD = 256;
-constexpr long long SMALL_BATCH_MAX_FLOATS = 20LL << 20;   // 80 MB of weights: they stay in the 126 MB L2 across iterations
+constexpr long long SMALL_MAX_FLOATS = 20LL << 20;   // 80 MB of weights: they stay in the 126 MB L2 across iterations
 constexpr int SMALL_CHUNK_ROWS = 32;   // threads with more rows than this move their fp32 sums out every 32 rows
 constexpr int SMALL_MIN_ROWS_PER_THREAD = 4;
 constexpr long long SMALL_SPIN_LIMIT = 2000000000LL;   // about a second of SM clock ticks per barrier wait
@@ -510,10 +512,11 @@ static int try_small_loop(idkm_ctx* ctx, const WorkspaceLayout& wl, const PassPa
   const int L = ctx->n_layers;
   const long long m = ctx->m_total;
   if (L > nb || L > MAX_LAYERS) return 1;
-  if (m > (long long)(L == 1 ? SMALL_ROWS_PER_THREAD : SMALL_BATCH_ROWS_PER_THREAD) * nb * BLOCK) return 1;
-  // (a batch whose weights do not stay in L2 is faster by a launch per iteration, whose kernels keep more loads in
-  // flight: 16 x 1 M rows at d = 2, k = 2: 68 against 38 us per iteration; 8 x 1 M at d = 4, k = 2: 65 against 41 us)
-  if (L > 1 && m * ctx->d > SMALL_BATCH_MAX_FLOATS) return 1;
+  const int per_thread = L > 1 ? SMALL_BATCH_ROWS_PER_THREAD : (ctx->d == 4 ? SMALL_ROWS_PER_THREAD_D4 : SMALL_ROWS_PER_THREAD);
+  if (m > (long long)per_thread * nb * BLOCK) return 1;
+  // (weights that do not stay in L2 are faster by a launch per iteration, whose kernels keep more loads in flight:
+  // 16 x 1 M rows at d = 2, k = 2: 68 against 38 us per iteration; 8 x 1 M at d = 4, k = 2: 65 against 41 us)
+  if (m * ctx->d > SMALL_MAX_FLOATS) return 1;
   long long grid = (m + (long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK - 1) / ((long long)SMALL_MIN_ROWS_PER_THREAD * BLOCK);
   if (grid > nb) grid = nb;
   if (grid < L) grid = L;
