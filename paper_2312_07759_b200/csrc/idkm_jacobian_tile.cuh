@@ -10,6 +10,13 @@
 // ((k d / 16)^2 entries per thread).  Sums: fp32 per 64 weights, moved into a second fp32 level, fp64 across blocks.
 // This is the paper's own formulation (it iterates a k x k matrix, Section 4.2); it replaces adj_max_iter passes over
 // W by one, which pays as soon as the iteration runs more than a few tens of steps.
+//
+// k d = 16 (QT below) takes a denser arrangement, because there a lane-per-centroid producer leaves half the lanes idle
+// and a thread's corner of the matrix is a single entry (two shared loads per FMA): every thread computes the attention
+// row of ONE weight (all centroids in its registers, no cross-lane reduction) and parks X_i, Y_i; then the 16 x 16
+// matrix is sixteen 4 x 4 tiles, each taken by sixteen threads that split the batch's 256 weights among them (two
+// 128-bit shared loads per 16 FMAs).  The diagonal term Dg is folded in: for d = 4 a diagonal tile is one (j, j) block
+// and reads Z_i[(j,b)] = (A_ij - 1) n_ijb in place of Y_i; for d < 4 the producer sums P_ija n_ijb itself.
 #pragma once
 #include "idkm_kernels.cuh"
 
@@ -24,7 +31,11 @@ struct JacTileCfg {
   static constexpr int PLEN = KD * KD + NDG;
   static constexpr int BATCH = 32;             // weights per batch (four per warp)
   static constexpr int TILE = 256;             // rows per tile of the layer table
-  static constexpr int XY_FLOATS = 2 * BATCH * KD;
+  static constexpr bool QT = (KD == 16);       // thread-per-weight producer, 4 x 4 tiles (see above)
+  static constexpr int QB = 256;               // weights per batch on that path (one per thread)
+  static constexpr int XS = 20;                // row stride of X / Y / Z there: 128-bit stores of consecutive rows hit
+                                               // different banks
+  static constexpr int XY_FLOATS = QT ? QB * XS * (D == 4 ? 3 : 2) : 2 * BATCH * KD;
   // dynamic shared memory: the X / Y batch while accumulating, the matrix (fp64) + u + g while solving
   static constexpr int SOLVE_BYTES = (KD * KD + 2 * KD) * 8;
   static constexpr int DYN_SMEM = (XY_FLOATS * 4 > SOLVE_BYTES ? XY_FLOATS * 4 : SOLVE_BYTES) + NDG * NWARP * 4;
@@ -35,9 +46,11 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
   using Cfg = JacTileCfg<D, KP>;
   constexpr int KD = Cfg::KD, TR = Cfg::TR, CPL = Cfg::CPL, NDG = Cfg::NDG, PLEN = Cfg::PLEN, BATCH = Cfg::BATCH;
   constexpr int TILE = Cfg::TILE;
+  constexpr bool QT = Cfg::QT;
+  constexpr int XS = Cfg::XS, QB = Cfg::QB;
   extern __shared__ __align__(16) unsigned char dyn[];
-  float* Xs = reinterpret_cast<float*>(dyn);              // [BATCH][KD]
-  float* Ys = Xs + BATCH * KD;                             // [BATCH][KD]
+  float* Xs = reinterpret_cast<float*>(dyn);              // [BATCH][KD]  (QT: [QB][XS])
+  float* Ys = Xs + (QT ? QB * XS : BATCH * KD);            // [BATCH][KD]  (QT: [QB][XS], then Z for d = 4)
   float* dgs = reinterpret_cast<float*>(dyn + (Cfg::DYN_SMEM - NDG * NWARP * 4));   // [NWARP][NDG]
   __shared__ int s_flag;
 
@@ -56,6 +69,12 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
   float dg[CPL][D][D], dg_hi[CPL][D][D];
   // consumer state: this thread's TR x TR corner of -X^T Y
   float acc[TR][TR], acc_hi[TR][TR];
+  // QT: all centroids of the layer in every thread; this thread's share of a 4 x 4 tile; the diagonal sums for d < 4
+  constexpr int NDQ = (QT && D < 4) ? KP * D * D : 1;
+  float cq[QT ? KP : 1][D], fq[QT ? KP : 1][D], iq[QT ? KP : 1];
+  float acc4[4][4], acc4_hi[4][4], dgt[NDQ], dgt_hi[NDQ];
+  (void)cq; (void)fq; (void)iq; (void)acc4; (void)acc4_hi; (void)dgt; (void)dgt_hi;
+  const int q_tile = tid >> 4, q_sub = tid & 15, q_ty = q_tile >> 2, q_tx = q_tile & 3;
   int layer = 0;
   while (p.lt.tile_off[layer + 1] <= t_lo) ++layer;
   int cur_layer = -1;
@@ -65,6 +84,30 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
   auto finish = [&](int l) {
     // ---- this block's partial: the matrix entries straight from their owners, the diagonal blocks over the warps
     double* mine = p.partials + (size_t)(b + l) * PLEN;
+    if constexpr (QT) {
+      // the sixteen threads of a tile (a half-warp) add their shares; the first writes the tile
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          float v = acc4_hi[i][j] + acc4[i][j];
+#pragma unroll
+          for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (q_sub == 0) mine[(q_ty * 4 + i) * KD + q_tx * 4 + j] = (double)v;
+        }
+      __syncthreads();   // the X / Y batch is no longer read
+      if constexpr (D < 4) {
+#pragma unroll
+        for (int o2 = 0; o2 < NDQ; ++o2) {
+          float v = dgt_hi[o2] + dgt[o2];
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          if (lane == 0) dgs[warp * NDG + o2] = v;
+        }
+      } else {
+        for (int o2 = lane; o2 < NDG; o2 += 32) dgs[warp * NDG + o2] = 0.f;   // (Dg is inside the diagonal tiles)
+      }
+    } else {
 #pragma unroll
     for (int i = 0; i < TR; ++i)
 #pragma unroll
@@ -80,6 +123,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
           const int j = lane + 32 * t;
           if (j < KP) dgs[warp * NDG + (j * D + a) * D + bb] = dg_hi[t][a][bb] + dg[t][a][bb];
         }
+    }
     __syncthreads();
     for (int o = tid; o < NDG; o += BLOCK) {
       double s = 0.0;
@@ -253,12 +297,145 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
             acc[i][j] = 0.f;
             acc_hi[i][j] = 0.f;
           }
+        if constexpr (QT) {
+#pragma unroll
+          for (int t = 0; t < KP; ++t) {
+            const bool ok = (t < k);
+            const float sv = ok ? p.S[(size_t)layer * k + t] : 0.f;
+            iq[t] = (ok && sv >= S_MIN_F) ? p.inv_tau / sv : 0.f;
+#pragma unroll
+            for (int a = 0; a < D; ++a) {
+              cq[t][a] = ok ? p.C[((size_t)layer * k + t) * D + a] : PAD_COORD;
+              fq[t][a] = ok ? p.F[((size_t)layer * k + t) * D + a] : 0.f;
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              acc4[i][j] = 0.f;
+              acc4_hi[i][j] = 0.f;
+            }
+#pragma unroll
+          for (int o2 = 0; o2 < NDQ; ++o2) {
+            dgt[o2] = 0.f;
+            dgt_hi[o2] = 0.f;
+          }
+        }
       }
     }
     if (!layer_active) continue;
     const long long row0 = p.lt.row_off[layer];
     const long long rows = p.lt.row_off[layer + 1] - row0;
     const long long tbase = (long long)(tile - p.lt.tile_off[layer]) * TILE;
+    if constexpr (QT) {
+      static_assert(!QT || TILE == QB, "one batch of the thread-per-weight path is one tile");
+      __syncthreads();   // the previous batch has been consumed
+      {
+        // ---- producer: this thread's weight of the batch ----
+        const long long loc = tbase + tid;
+        const bool valid = (loc < rows);
+        const long long grow = row0 + (valid ? loc : 0);
+        float w[D];
+        if constexpr (D == 4) {
+          const float4 x = __ldg(reinterpret_cast<const float4*>(p.W + grow * 4));
+          w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
+        } else if constexpr (D == 2) {
+          const float2 x = __ldg(reinterpret_cast<const float2*>(p.W + grow * 2));
+          w[0] = x.x; w[1] = x.y;
+        } else {
+          w[0] = __ldg(p.W + grow);
+        }
+        float e[KP], rsq[D > 1 ? KP : 1];
+        (void)rsq;
+        float lmin = 3.0e38f;
+#pragma unroll
+        for (int t = 0; t < KP; ++t) {
+          if constexpr (D == 1) {
+            e[t] = fabsf(w[0] - cq[t][0]);
+          } else {
+            float sq = 1e-30f;
+#pragma unroll
+            for (int a = 0; a < D; ++a) {
+              const float df = w[a] - cq[t][a];
+              sq = fmaf(df, df, sq);
+            }
+            rsq[t] = rsqrt_approx(sq);
+            e[t] = sq * rsq[t];
+          }
+          lmin = fminf(lmin, e[t]);
+        }
+        const float mref = lmin * p.scale;
+        float lsum = 0.f;
+#pragma unroll
+        for (int t = 0; t < KP; ++t) {
+          e[t] = ex2_approx(fmaf(-p.scale, e[t], mref));
+          lsum += e[t];
+        }
+        const float rr = valid ? rcp_approx(lsum) : 0.f;
+        float xr[KD], yr[KD], zr[D == 4 ? KD : 1];
+        (void)zr;
+#pragma unroll
+        for (int t = 0; t < KP; ++t) {
+          const float at = e[t] * rr;
+          float nn[D], pp[D];
+#pragma unroll
+          for (int a = 0; a < D; ++a) {
+            const float df = w[a] - cq[t][a];
+            if constexpr (D == 1) nn[a] = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
+            else nn[a] = df * rsq[t];
+            pp[a] = at * iq[t] * (w[a] - fq[t][a]);
+            xr[t * D + a] = pp[a];
+            yr[t * D + a] = at * nn[a];
+            if constexpr (D == 4) zr[t * D + a] = (at - 1.f) * nn[a];
+          }
+          if constexpr (D < 4) {
+#pragma unroll
+            for (int a = 0; a < D; ++a)
+#pragma unroll
+              for (int bb = 0; bb < D; ++bb) dgt[(t * D + a) * D + bb] = fmaf(pp[a], nn[bb], dgt[(t * D + a) * D + bb]);
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < KD / 4; ++q) {
+          *reinterpret_cast<float4*>(Xs + tid * XS + 4 * q) = make_float4(xr[4 * q], xr[4 * q + 1], xr[4 * q + 2], xr[4 * q + 3]);
+          *reinterpret_cast<float4*>(Ys + tid * XS + 4 * q) = make_float4(yr[4 * q], yr[4 * q + 1], yr[4 * q + 2], yr[4 * q + 3]);
+          if constexpr (D == 4)
+            *reinterpret_cast<float4*>(Ys + QB * XS + tid * XS + 4 * q) = make_float4(zr[4 * q], zr[4 * q + 1], zr[4 * q + 2], zr[4 * q + 3]);
+        }
+      }
+      __syncthreads();
+      {
+        // ---- consumer: this thread's sixteenth of the batch into its 4 x 4 tile ----
+        const float* ysrc = (D == 4 && q_ty == q_tx) ? Ys + QB * XS : Ys;
+#pragma unroll 4
+        for (int r = q_sub; r < QB; r += 16) {
+          const float4 x4 = *reinterpret_cast<const float4*>(Xs + r * XS + 4 * q_ty);
+          const float4 y4 = *reinterpret_cast<const float4*>(ysrc + r * XS + 4 * q_tx);
+          const float xv[4] = {x4.x, x4.y, x4.z, x4.w}, yv[4] = {y4.x, y4.y, y4.z, y4.w};
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc4[i][j] = fmaf(-xv[i], yv[j], acc4[i][j]);
+        }
+        if (++batches == 4) {   // 64 weights per thread: move the sums to the second level
+#pragma unroll
+          for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              acc4_hi[i][j] += acc4[i][j];
+              acc4[i][j] = 0.f;
+            }
+#pragma unroll
+          for (int o2 = 0; o2 < NDQ; ++o2) {
+            dgt_hi[o2] += dgt[o2];
+            dgt[o2] = 0.f;
+          }
+          batches = 0;
+        }
+      }
+      continue;
+    }
 #pragma unroll 1
     for (int b0 = 0; b0 < TILE; b0 += BATCH) {
       if (tbase + b0 >= rows) break;   // uniform over the block
