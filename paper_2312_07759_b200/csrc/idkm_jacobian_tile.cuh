@@ -11,12 +11,13 @@
 // This is the paper's own formulation (it iterates a k x k matrix, Section 4.2); it replaces adj_max_iter passes over
 // W by one, which pays as soon as the iteration runs more than a few tens of steps.
 //
-// k d = 16 (QT below) takes a denser arrangement, because there a lane-per-centroid producer leaves half the lanes idle
-// and a thread's corner of the matrix is a single entry (two shared loads per FMA): every thread computes the attention
-// row of ONE weight (all centroids in its registers, no cross-lane reduction) and parks X_i, Y_i; then the 16 x 16
-// matrix is sixteen 4 x 4 tiles, each taken by sixteen threads that split the batch's 256 weights among them (two
-// 128-bit shared loads per 16 FMAs).  The diagonal term Dg is folded in: for d = 4 a diagonal tile is one (j, j) block
-// and reads Z_i[(j,b)] = (A_ij - 1) n_ijb in place of Y_i; for d < 4 the producer sums P_ija n_ijb itself.
+// k d = 16 and 32 (QT below) take a denser arrangement, because there a lane-per-centroid producer leaves lanes idle
+// and a thread's corner of the matrix is one or four entries (one shared load per FMA): a thread computes the attention
+// row of ONE weight (no cross-lane reduction; the centroids in its registers at k d = 16, in shared memory at 32) and
+// parks X_i, Y_i; then the matrix is (k d / 4)^2 tiles of 4 x 4, each taken by 16 resp. 4 threads that split the
+// batch's weights among them (two 128-bit shared loads per 16 FMAs).  The diagonal term Dg is folded in: the producer
+// also parks Z_i[(j,b)] = (A_ij - 1) n_ijb and the entries of a diagonal tile that belong to a (j, j) block take Z_i in
+// place of Y_i (at d = 4 that is the whole tile); at k d = 16 with d < 4 the producer sums P_ija n_ijb itself instead.
 #pragma once
 #include "idkm_kernels.cuh"
 
@@ -31,11 +32,15 @@ struct JacTileCfg {
   static constexpr int PLEN = KD * KD + NDG;
   static constexpr int BATCH = 32;             // weights per batch (four per warp)
   static constexpr int TILE = 256;             // rows per tile of the layer table
-  static constexpr bool QT = (KD == 16);       // thread-per-weight producer, 4 x 4 tiles (see above)
-  static constexpr int QB = 256;               // weights per batch on that path (one per thread)
-  static constexpr int XS = 20;                // row stride of X / Y / Z there: 128-bit stores of consecutive rows hit
-                                               // different banks
-  static constexpr int XY_FLOATS = QT ? QB * XS * (D == 4 ? 3 : 2) : 2 * BATCH * KD;
+  static constexpr bool QT = (KD == 16 || KD == 32);   // thread-per-weight producer, 4 x 4 tiles (see above)
+  static constexpr bool QREG = (KD == 16);             // ... with the centroids in registers (else in shared memory)
+  static constexpr bool QZ = QT && (D == 4 || KD == 32);   // ... with Z rows (else the producer sums Dg)
+  static constexpr int QB = (KD == 16) ? 256 : 128;    // weights per batch on that path (one per producing thread)
+  static constexpr int XS = KD + 4;                    // row stride of X / Y / Z there: 128-bit stores of consecutive
+                                                       // rows hit different banks
+  static constexpr int NT1 = KD / 4;                   // tiles per side
+  static constexpr int TPT = QT ? BLOCK / (NT1 * NT1) : 1;   // threads per tile
+  static constexpr int XY_FLOATS = QT ? QB * XS * (QZ ? 3 : 2) : 2 * BATCH * KD;
   // dynamic shared memory: the X / Y batch while accumulating, the matrix (fp64) + u + g while solving
   static constexpr int SOLVE_BYTES = (KD * KD + 2 * KD) * 8;
   static constexpr int DYN_SMEM = (XY_FLOATS * 4 > SOLVE_BYTES ? XY_FLOATS * 4 : SOLVE_BYTES) + NDG * NWARP * 4;
@@ -46,8 +51,8 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
   using Cfg = JacTileCfg<D, KP>;
   constexpr int KD = Cfg::KD, TR = Cfg::TR, CPL = Cfg::CPL, NDG = Cfg::NDG, PLEN = Cfg::PLEN, BATCH = Cfg::BATCH;
   constexpr int TILE = Cfg::TILE;
-  constexpr bool QT = Cfg::QT;
-  constexpr int XS = Cfg::XS, QB = Cfg::QB;
+  constexpr bool QT = Cfg::QT, QREG = Cfg::QREG, QZ = Cfg::QZ;
+  constexpr int XS = Cfg::XS, QB = Cfg::QB, NT1 = Cfg::NT1, TPT = Cfg::TPT;
   extern __shared__ __align__(16) unsigned char dyn[];
   float* Xs = reinterpret_cast<float*>(dyn);              // [BATCH][KD]  (QT: [QB][XS])
   float* Ys = Xs + (QT ? QB * XS : BATCH * KD);            // [BATCH][KD]  (QT: [QB][XS], then Z for d = 4)
@@ -69,12 +74,17 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
   float dg[CPL][D][D], dg_hi[CPL][D][D];
   // consumer state: this thread's TR x TR corner of -X^T Y
   float acc[TR][TR], acc_hi[TR][TR];
-  // QT: all centroids of the layer in every thread; this thread's share of a 4 x 4 tile; the diagonal sums for d < 4
-  constexpr int NDQ = (QT && D < 4) ? KP * D * D : 1;
-  float cq[QT ? KP : 1][D], fq[QT ? KP : 1][D], iq[QT ? KP : 1];
+  // QT: all centroids of the layer in every thread (or in shared memory); this thread's share of a 4 x 4 tile; the
+  // diagonal sums where the producer keeps them
+  constexpr int NDQ = (QT && !QZ) ? KP * D * D : 1;
+  float cq[QREG ? KP : 1][D], fq[QREG ? KP : 1][D], iq[QREG ? KP : 1];
+  __shared__ float c_s[(QT && !QREG) ? KP * D : 1], f_s[(QT && !QREG) ? KP * D : 1], i_s[(QT && !QREG) ? KP : 1];
   float acc4[4][4], acc4_hi[4][4], dgt[NDQ], dgt_hi[NDQ];
-  (void)cq; (void)fq; (void)iq; (void)acc4; (void)acc4_hi; (void)dgt; (void)dgt_hi;
-  const int q_tile = tid >> 4, q_sub = tid & 15, q_ty = q_tile >> 2, q_tx = q_tile & 3;
+  (void)cq; (void)fq; (void)iq; (void)acc4; (void)acc4_hi; (void)dgt; (void)dgt_hi; (void)c_s; (void)f_s; (void)i_s;
+  auto cget = [&](int t, int a) -> float { return QREG ? cq[QREG ? t : 0][a] : c_s[(QT && !QREG) ? t * D + a : 0]; };
+  auto fget = [&](int t, int a) -> float { return QREG ? fq[QREG ? t : 0][a] : f_s[(QT && !QREG) ? t * D + a : 0]; };
+  auto iget = [&](int t) -> float { return QREG ? iq[QREG ? t : 0] : i_s[(QT && !QREG) ? t : 0]; };
+  const int q_tile = tid / TPT, q_sub = tid % TPT, q_ty = q_tile / NT1, q_tx = q_tile % NT1;
   int layer = 0;
   while (p.lt.tile_off[layer + 1] <= t_lo) ++layer;
   int cur_layer = -1;
@@ -85,18 +95,18 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
     // ---- this block's partial: the matrix entries straight from their owners, the diagonal blocks over the warps
     double* mine = p.partials + (size_t)(b + l) * PLEN;
     if constexpr (QT) {
-      // the sixteen threads of a tile (a half-warp) add their shares; the first writes the tile
+      // the threads of a tile (neighbouring lanes) add their shares; the first writes the tile
 #pragma unroll
       for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           float v = acc4_hi[i][j] + acc4[i][j];
 #pragma unroll
-          for (int o = 8; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+          for (int o = TPT / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
           if (q_sub == 0) mine[(q_ty * 4 + i) * KD + q_tx * 4 + j] = (double)v;
         }
       __syncthreads();   // the X / Y batch is no longer read
-      if constexpr (D < 4) {
+      if constexpr (!QZ) {
 #pragma unroll
         for (int o2 = 0; o2 < NDQ; ++o2) {
           float v = dgt_hi[o2] + dgt[o2];
@@ -298,15 +308,29 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
             acc_hi[i][j] = 0.f;
           }
         if constexpr (QT) {
+          if constexpr (QREG) {
 #pragma unroll
-          for (int t = 0; t < KP; ++t) {
-            const bool ok = (t < k);
-            const float sv = ok ? p.S[(size_t)layer * k + t] : 0.f;
-            iq[t] = (ok && sv >= S_MIN_F) ? p.inv_tau / sv : 0.f;
+            for (int t = 0; t < KP; ++t) {
+              const bool ok = (t < k);
+              const float sv = ok ? p.S[(size_t)layer * k + t] : 0.f;
+              iq[t] = (ok && sv >= S_MIN_F) ? p.inv_tau / sv : 0.f;
 #pragma unroll
-            for (int a = 0; a < D; ++a) {
-              cq[t][a] = ok ? p.C[((size_t)layer * k + t) * D + a] : PAD_COORD;
-              fq[t][a] = ok ? p.F[((size_t)layer * k + t) * D + a] : 0.f;
+              for (int a = 0; a < D; ++a) {
+                cq[t][a] = ok ? p.C[((size_t)layer * k + t) * D + a] : PAD_COORD;
+                fq[t][a] = ok ? p.F[((size_t)layer * k + t) * D + a] : 0.f;
+              }
+            }
+          } else {
+            // (finish() of the previous layer ended with a barrier; the batch body starts with one)
+            for (int o2 = tid; o2 < KP * D; o2 += BLOCK) {
+              const bool ok = (o2 / D < k);
+              c_s[o2] = ok ? p.C[(size_t)layer * k * D + o2] : PAD_COORD;
+              f_s[o2] = ok ? p.F[(size_t)layer * k * D + o2] : 0.f;
+            }
+            for (int t = tid; t < KP; t += BLOCK) {
+              const bool ok = (t < k);
+              const float sv = ok ? p.S[(size_t)layer * k + t] : 0.f;
+              i_s[t] = (ok && sv >= S_MIN_F) ? p.inv_tau / sv : 0.f;
             }
           }
 #pragma unroll
@@ -329,109 +353,125 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_jacobian_tile(const __grid_cons
     const long long rows = p.lt.row_off[layer + 1] - row0;
     const long long tbase = (long long)(tile - p.lt.tile_off[layer]) * TILE;
     if constexpr (QT) {
-      static_assert(!QT || TILE == QB, "one batch of the thread-per-weight path is one tile");
-      __syncthreads();   // the previous batch has been consumed
-      {
-        // ---- producer: this thread's weight of the batch ----
-        const long long loc = tbase + tid;
-        const bool valid = (loc < rows);
-        const long long grow = row0 + (valid ? loc : 0);
-        float w[D];
-        if constexpr (D == 4) {
-          const float4 x = __ldg(reinterpret_cast<const float4*>(p.W + grow * 4));
-          w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
-        } else if constexpr (D == 2) {
-          const float2 x = __ldg(reinterpret_cast<const float2*>(p.W + grow * 2));
-          w[0] = x.x; w[1] = x.y;
-        } else {
-          w[0] = __ldg(p.W + grow);
-        }
-        float e[KP], rsq[D > 1 ? KP : 1];
-        (void)rsq;
-        float lmin = 3.0e38f;
-#pragma unroll
-        for (int t = 0; t < KP; ++t) {
-          if constexpr (D == 1) {
-            e[t] = fabsf(w[0] - cq[t][0]);
+      static_assert(!QT || TILE % QB == 0, "a tile of the layer table is a whole number of batches");
+#pragma unroll 1
+      for (int b0 = 0; b0 < TILE; b0 += QB) {
+        if (tbase + b0 >= rows) break;   // uniform over the block
+        __syncthreads();   // the previous batch has been consumed (and the layer's constants are in place)
+        if (tid < QB) {
+          // ---- producer: this thread's weight of the batch ----
+          const long long loc = tbase + b0 + tid;
+          const bool valid = (loc < rows);
+          const long long grow = row0 + (valid ? loc : 0);
+          float w[D];
+          if constexpr (D == 4) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(p.W + grow * 4));
+            w[0] = x.x; w[1] = x.y; w[2] = x.z; w[3] = x.w;
+          } else if constexpr (D == 2) {
+            const float2 x = __ldg(reinterpret_cast<const float2*>(p.W + grow * 2));
+            w[0] = x.x; w[1] = x.y;
           } else {
-            float sq = 1e-30f;
+            w[0] = __ldg(p.W + grow);
+          }
+          float e[KP], rsq[D > 1 ? KP : 1];
+          (void)rsq;
+          float lmin = 3.0e38f;
 #pragma unroll
-            for (int a = 0; a < D; ++a) {
-              const float df = w[a] - cq[t][a];
-              sq = fmaf(df, df, sq);
+          for (int t = 0; t < KP; ++t) {
+            if constexpr (D == 1) {
+              e[t] = fabsf(w[0] - cget(t, 0));
+            } else {
+              float sq = 1e-30f;
+#pragma unroll
+              for (int a = 0; a < D; ++a) {
+                const float df = w[a] - cget(t, a);
+                sq = fmaf(df, df, sq);
+              }
+              rsq[t] = rsqrt_approx(sq);
+              e[t] = sq * rsq[t];
             }
-            rsq[t] = rsqrt_approx(sq);
-            e[t] = sq * rsq[t];
+            lmin = fminf(lmin, e[t]);
           }
-          lmin = fminf(lmin, e[t]);
-        }
-        const float mref = lmin * p.scale;
-        float lsum = 0.f;
+          const float mref = lmin * p.scale;
+          float lsum = 0.f;
 #pragma unroll
-        for (int t = 0; t < KP; ++t) {
-          e[t] = ex2_approx(fmaf(-p.scale, e[t], mref));
-          lsum += e[t];
-        }
-        const float rr = valid ? rcp_approx(lsum) : 0.f;
-        float xr[KD], yr[KD], zr[D == 4 ? KD : 1];
-        (void)zr;
-#pragma unroll
-        for (int t = 0; t < KP; ++t) {
-          const float at = e[t] * rr;
-          float nn[D], pp[D];
-#pragma unroll
-          for (int a = 0; a < D; ++a) {
-            const float df = w[a] - cq[t][a];
-            if constexpr (D == 1) nn[a] = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
-            else nn[a] = df * rsq[t];
-            pp[a] = at * iq[t] * (w[a] - fq[t][a]);
-            xr[t * D + a] = pp[a];
-            yr[t * D + a] = at * nn[a];
-            if constexpr (D == 4) zr[t * D + a] = (at - 1.f) * nn[a];
+          for (int t = 0; t < KP; ++t) {
+            e[t] = ex2_approx(fmaf(-p.scale, e[t], mref));
+            lsum += e[t];
           }
-          if constexpr (D < 4) {
+          const float rr = valid ? rcp_approx(lsum) : 0.f;
+          // four consecutive entries of the rows at a time (4 / D centroids), stored as soon as they are complete
+          constexpr int CPC = 4 / D;
 #pragma unroll
-            for (int a = 0; a < D; ++a)
+          for (int q = 0; q < KD / 4; ++q) {
+            float xv[4], yv[4], zv[4];
+            (void)zv;
 #pragma unroll
-              for (int bb = 0; bb < D; ++bb) dgt[(t * D + a) * D + bb] = fmaf(pp[a], nn[bb], dgt[(t * D + a) * D + bb]);
+            for (int cc = 0; cc < CPC; ++cc) {
+              const int t = q * CPC + cc;
+              const float at = e[t] * rr;
+              float nn[D], pp[D];
+#pragma unroll
+              for (int a = 0; a < D; ++a) {
+                const float df = w[a] - cget(t, a);
+                if constexpr (D == 1) nn[a] = (df > 0.f) ? 1.f : ((df < 0.f) ? -1.f : 0.f);
+                else nn[a] = df * rsq[t];
+                pp[a] = at * iget(t) * (w[a] - fget(t, a));
+                xv[cc * D + a] = pp[a];
+                yv[cc * D + a] = at * nn[a];
+                zv[cc * D + a] = (at - 1.f) * nn[a];
+              }
+              if constexpr (!QZ) {
+#pragma unroll
+                for (int a = 0; a < D; ++a)
+#pragma unroll
+                  for (int bb = 0; bb < D; ++bb)
+                    dgt[(t * D + a) * D + bb] = fmaf(pp[a], nn[bb], dgt[(t * D + a) * D + bb]);
+              }
+            }
+            *reinterpret_cast<float4*>(Xs + tid * XS + 4 * q) = make_float4(xv[0], xv[1], xv[2], xv[3]);
+            *reinterpret_cast<float4*>(Ys + tid * XS + 4 * q) = make_float4(yv[0], yv[1], yv[2], yv[3]);
+            if constexpr (QZ) *reinterpret_cast<float4*>(Ys + QB * XS + tid * XS + 4 * q) = make_float4(zv[0], zv[1], zv[2], zv[3]);
           }
         }
-#pragma unroll
-        for (int q = 0; q < KD / 4; ++q) {
-          *reinterpret_cast<float4*>(Xs + tid * XS + 4 * q) = make_float4(xr[4 * q], xr[4 * q + 1], xr[4 * q + 2], xr[4 * q + 3]);
-          *reinterpret_cast<float4*>(Ys + tid * XS + 4 * q) = make_float4(yr[4 * q], yr[4 * q + 1], yr[4 * q + 2], yr[4 * q + 3]);
-          if constexpr (D == 4)
-            *reinterpret_cast<float4*>(Ys + QB * XS + tid * XS + 4 * q) = make_float4(zr[4 * q], zr[4 * q + 1], zr[4 * q + 2], zr[4 * q + 3]);
-        }
-      }
-      __syncthreads();
-      {
-        // ---- consumer: this thread's sixteenth of the batch into its 4 x 4 tile ----
-        const float* ysrc = (D == 4 && q_ty == q_tx) ? Ys + QB * XS : Ys;
+        __syncthreads();
+        {
+          // ---- consumer: this thread's share of the batch into its 4 x 4 tile ----
+          const bool diag = (q_ty == q_tx);
+          const float* ysrc = (QZ && D == 4 && diag) ? Ys + QB * XS : Ys;
 #pragma unroll 4
-        for (int r = q_sub; r < QB; r += 16) {
-          const float4 x4 = *reinterpret_cast<const float4*>(Xs + r * XS + 4 * q_ty);
-          const float4 y4 = *reinterpret_cast<const float4*>(ysrc + r * XS + 4 * q_tx);
-          const float xv[4] = {x4.x, x4.y, x4.z, x4.w}, yv[4] = {y4.x, y4.y, y4.z, y4.w};
+          for (int r = q_sub; r < QB; r += TPT) {
+            const float4 x4 = *reinterpret_cast<const float4*>(Xs + r * XS + 4 * q_ty);
+            const float4 y4 = *reinterpret_cast<const float4*>(ysrc + r * XS + 4 * q_tx);
+            const float xv[4] = {x4.x, x4.y, x4.z, x4.w}, yv[4] = {y4.x, y4.y, y4.z, y4.w};
+            float ys[4] = {yv[0], yv[1], yv[2], yv[3]};   // what the entries of a (j, j) block multiply
+            if constexpr (QZ && D < 4) {
+              const float4 z4 = *reinterpret_cast<const float4*>(Ys + QB * XS + r * XS + 4 * q_tx);
+              const float zv[4] = {z4.x, z4.y, z4.z, z4.w};
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) acc4[i][j] = fmaf(-xv[i], yv[j], acc4[i][j]);
-        }
-        if (++batches == 4) {   // 64 weights per thread: move the sums to the second level
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              acc4_hi[i][j] += acc4[i][j];
-              acc4[i][j] = 0.f;
+              for (int j = 0; j < 4; ++j) ys[j] = diag ? zv[j] : yv[j];
             }
 #pragma unroll
-          for (int o2 = 0; o2 < NDQ; ++o2) {
-            dgt_hi[o2] += dgt[o2];
-            dgt[o2] = 0.f;
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) acc4[i][j] = fmaf(-xv[i], (i / D == j / D) ? ys[j] : yv[j], acc4[i][j]);
           }
-          batches = 0;
+          // every 64 weights of this thread: move the sums to the second level
+          if (++batches == (64 * TPT) / QB) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                acc4_hi[i][j] += acc4[i][j];
+                acc4[i][j] = 0.f;
+              }
+#pragma unroll
+            for (int o2 = 0; o2 < NDQ; ++o2) {
+              dgt_hi[o2] += dgt[o2];
+              dgt[o2] = 0.f;
+            }
+            batches = 0;
+          }
         }
       }
       continue;
