@@ -94,6 +94,8 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
   const float inv_tau = (float)sp.inv_tau_d;
   const float inv_k = 1.f / (float)k;
   bool ok = true;
+  // a grid of one block (a layer of a few thousand weights) needs neither the partial buffers nor the barrier
+  const bool solo = (G == 1) && (sp.missing_arrivals == 0);
 
   for (int it = 0; it < sp.max_iter; ++it) {
     if (sp.n_layers == 1 && done) break;   // (a batch goes on meeting at the barrier until every layer has ended)
@@ -308,12 +310,17 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
       double s = 0.0;
 #pragma unroll
       for (int wv = 0; wv < NWARP; ++wv) s += (double)red[wv][tid];
-      __stcg(mine + tid, s);
+      if (solo) tot[tid] = s;   // a grid of one block: the layer's totals, no trip through global memory
+      else __stcg(mine + tid, s);
     }
     }   // !done
+    if (solo) {
+      __syncthreads();
+    } else {
     // ---- everyone has published: grid-wide barrier ----
     ok = small_barrier(sp.sync, (unsigned int)(it + 1) * (unsigned int)(G + sp.missing_arrivals), sp.spin_limit, &s_ok);
     if (!ok) break;
+    }
     // A batch ends at the first barrier at which every layer's loop has ended: the first block of a layer publishes
     // fwd_done = (iterations taken) before it arrives at the next barrier, so after barrier `it` every value in
     // (0, it] is final and seen by all blocks alike; a later value cannot be mistaken for one of them.
@@ -327,7 +334,7 @@ __global__ void __launch_bounds__(BLOCK, 2) idkm_small_loop(const __grid_constan
     }
     if (done) continue;
     // ---- every block of the layer adds the layer's partials in the same order ----
-    {
+    if (!solo) {
       const double* base = sp.partials + ((size_t)(it & 1) * G + first_blk) * PLEN;
       const int ch = tid / PLEN, o = tid % PLEN;
       if (ch < CH) {
